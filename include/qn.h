@@ -1,0 +1,159 @@
+/*
+ * qn.h -- C ABI of the B200 (sm_100a) Parameter-Server quasi-Newton step of Arnold & Wang,
+ * "Accelerating SGD for Distributed Deep-Learning Using Approximated Hessian Matrix"
+ * (arXiv 1709.05069), Section 2 (Method).
+ *
+ * What one call computes (Section 2, Eq. (2)-(4)).  Given m Workers' parameter vectors
+ * theta_k in R^n and gradients g_k = grad J(theta_k):
+ *     gbar, thetabar      means over the Workers                         (display before Eq. (2))
+ *     G, Theta            n x m, columns g_k - gbar and theta_k - thetabar
+ *     G^T G = V diag(sigma^2) V^T,  sigma_1 >= ... >= sigma_m >= 0       (SVD paragraph)
+ *     j                   sigma_j >= lambda sigma_1 > sigma_{j+1}        (text after Eq. (3))
+ *     u_k = G v_k / ||G v_k||,  y_k = Theta v_k,  alpha_k = gbar^T u_k   (k = 1..j)
+ *     theta_new = thetabar - tau ( gbar - sum alpha_k u_k + sum alpha_k sigma_k^-1 y_k )   Eq. (2),(4)
+ * and j = 0 gives plain SGD, thetabar - tau gbar (sentence after Eq. (4)).
+ *
+ * Layout.  All matrices are Worker-major: theta[m][n] and g[m][n], row k = Worker k, each row
+ * contiguous (the transpose of the paper's n x m matrices).  Elements are fp32 or bf16
+ * (qn_dtype); all arithmetic is fp32 products with fp64 accumulation for the Gram, fp64 for the
+ * m x m eigen-problem and the coefficients, fp32 for the final combination, and one
+ * round-to-nearest-even to the storage type when theta_new is written.
+ *
+ * Pointers.  Unless a parameter says HOST, data pointers are DEVICE pointers on the device that
+ * was current when the handle was created.  The caller owns every buffer it passes; the library
+ * only reads inputs and only writes the named outputs.  The handle owns its workspace.
+ * Rows that start on 16-byte boundaries (base pointer 16-byte aligned and n * element size a
+ * multiple of 16) take the vectorised path; anything else takes a slower element-wise path,
+ * never an error.
+ *
+ * Streams.  `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ * Calls enqueue work on that stream and return without waiting unless they have to hand a HOST
+ * result back (j_out / sigma_out non-NULL, qn_status_sync, qn_update_host).
+ *
+ * Errors.  Every call returns a qn_status; nothing throws or aborts.  Arguments are validated on
+ * the host before anything is launched.  Conditions only the device can see (a non-finite Gram,
+ * the Jacobi sweep limit) are recorded in a device status word that is returned by the next call
+ * that synchronises; in both cases theta_new is still written (with j = 0, i.e. the SGD update,
+ * for a non-finite Gram).
+ *
+ * There is no CPU fallback: without a usable CUDA device qn_create fails with QN_ERR_CUDA.
+ */
+#ifndef QN_H
+#define QN_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define QN_MAX_M 64 /* largest supported number of Workers */
+
+#if defined(__GNUC__)
+#define QN_API __attribute__((visibility("default")))
+#else
+#define QN_API
+#endif
+
+typedef struct qn_ctx* qn_handle;
+
+typedef enum { QN_F32 = 0, QN_BF16 = 1 } qn_dtype;
+
+typedef enum {
+    QN_OK = 0,
+    QN_ERR_INVALID = 1,       /* bad argument (null, n < 1, m outside [1, QN_MAX_M], lambda <= 0, ...) */
+    QN_ERR_ALLOC = 2,         /* device or host allocation failed */
+    QN_ERR_CUDA = 3,          /* a CUDA runtime call failed (no device, launch error, ...) */
+    QN_ERR_STATE = 4,         /* call not valid in the handle's state (window not full, ...) */
+    QN_ERR_NOT_CONVERGED = 5, /* Jacobi hit its sweep limit; results were still written */
+    QN_ERR_NONFINITE = 6      /* Gram contained NaN/Inf; theta_new written with j = 0 */
+} qn_status;
+
+/* Human-readable text for a status code (static storage, never NULL). */
+QN_API const char* qn_strerror(qn_status s);
+
+/*
+ * Create a handle for n parameters, m Workers and the given storage type on the CURRENT CUDA
+ * device, and allocate its workspace there (a few MB; the asynchronous window is allocated by
+ * the first qn_push).  1 <= m <= QN_MAX_M, n >= 1.  *out is set only on QN_OK.
+ */
+QN_API qn_status qn_create(int64_t n, int32_t m, qn_dtype dtype, qn_handle* out);
+
+/* Free the handle and everything it owns.  Waits for the device to finish work it enqueued. */
+QN_API qn_status qn_destroy(qn_handle h);
+
+/*
+ * Synchronous mode: the whole Server step (Section 2, Eq. (2)-(4)) on all m Workers at once.
+ *   theta, g     [m][n], read-only
+ *   tau          learning rate of Eq. (2), finite
+ *   lambda       cut-off of the text after Eq. (3); > 0 and finite.  0 < lambda < 1 is the paper's
+ *                range; lambda > 1 is accepted and keeps no mode (j = 0, the SGD update)
+ *   theta_new    [n], written; must not overlap the inputs
+ *   j_out        HOST int32, may be NULL
+ *   sigma_out    HOST double[m], descending, may be NULL
+ * If both j_out and sigma_out are NULL the call does not wait for the device.
+ */
+QN_API qn_status qn_update(qn_handle h, const void* theta, const void* g, double tau, double lambda,
+                    void* theta_new, int32_t* j_out, double* sigma_out, void* cuda_stream);
+
+/*
+ * The reductions alone: the centred Gram C = G^T G (m x m, row-major, symmetric) followed by
+ * w = G^T gbar (m values), as m*m + m doubles written to the DEVICE buffer gram_out
+ * (Section 2: the matrix G^H G of the SVD paragraph, and the numerators of alpha_k = z^H u_k
+ * for z = gbar).  The means and the centred columns are formed on the fly and never stored.
+ */
+QN_API qn_status qn_gram(qn_handle h, const void* g, double* gram_out, void* cuda_stream);
+
+/*
+ * Asynchronous mode (Section 2, first sentence: an update may follow each Write by one Worker).
+ * The handle keeps a window of the m most recent (theta, g) pairs and the raw m x m Gram of the
+ * window's gradients in fp64.  qn_push lands one Worker's Write in a slot and refreshes that
+ * slot's Gram row and column in O(m n); the paper is silent on which pair a Write replaces:
+ * slot = -1 replaces the oldest, 0 <= slot < m replaces that slot.
+ *   theta_col, g_col   [n] each, read-only
+ */
+QN_API qn_status qn_push(qn_handle h, int32_t slot, const void* theta_col, const void* g_col, void* cuda_stream);
+
+/*
+ * The Server step on the window's current contents.  QN_ERR_STATE until every slot has been
+ * written at least once.  Outputs as in qn_update.
+ */
+QN_API qn_status qn_update_window(qn_handle h, double tau, double lambda, void* theta_new, int32_t* j_out,
+                           double* sigma_out, void* cuda_stream);
+
+/* Recompute the window's raw Gram from its columns in O(m^2 n) (drift correction / after restore). */
+QN_API qn_status qn_rebuild(qn_handle h, void* cuda_stream);
+
+/*
+ * DEVICE pointers to the window's storage, [m][n] each, so that a caller can restore or inspect
+ * it (follow a restore with qn_rebuild and qn_window_mark_full).  NULL before the first qn_push
+ * unless qn_window_alloc was called.
+ */
+QN_API qn_status qn_window_alloc(qn_handle h);
+QN_API void* qn_window_theta(qn_handle h);
+QN_API void* qn_window_g(qn_handle h);
+QN_API qn_status qn_window_mark_full(qn_handle h);
+
+/*
+ * qn_update with HOST buffers: copies theta and g (HOST, [m][n], pinned memory recommended) to
+ * device staging owned by the handle, runs the step, copies theta_new back to theta_new_host
+ * ([n]) and waits.  The staging (2 m n + n elements) is allocated by the first call.
+ */
+QN_API qn_status qn_update_host(qn_handle h, const void* theta_host, const void* g_host, double tau, double lambda,
+                         void* theta_new_host, int32_t* j_out, double* sigma_out, void* cuda_stream);
+
+/* Wait for the stream last used with this handle and return the deferred device status. */
+QN_API qn_status qn_status_sync(qn_handle h);
+
+/* Number of kernels this handle launched in its most recent qn_* call, and since creation. */
+QN_API int32_t qn_last_launches(qn_handle h);
+QN_API int64_t qn_total_launches(qn_handle h);
+
+/* Jacobi sweeps used by the most recent step whose results were fetched to the host (j_out or
+ * sigma_out non-NULL, or qn_status_sync), else -1. */
+QN_API int32_t qn_last_sweeps(qn_handle h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QN_H */

@@ -1,0 +1,415 @@
+// C ABI of libqn: argument checks, workspace, launch sequences.  See include/qn.h for the contract.
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "qn_internal.h"
+
+struct qn_ctx {
+    int64_t n;
+    int32_t m;
+    qn_dtype dtype;
+    size_t elem;
+    int device;
+
+    double* partials;  // device, max_partials * qn_partial_len(m)
+    int max_partials;
+    qn_coef_block* coef;          // device
+    qn_result_block* result;      // device
+    qn_result_block* host_result; // pinned host
+    unsigned int* ticket;         // device, zero between launches
+
+    // asynchronous window
+    void* win_theta;
+    void* win_g;
+    double* raw_gram;  // device, m*m
+    uint64_t filled;   // bit k set once slot k has been written
+    int32_t head;      // slot of the oldest column
+
+    // host-buffer path
+    void* stage_theta;
+    void* stage_g;
+    void* stage_out;
+
+    cudaStream_t last_stream;
+    int32_t last_launches;
+    int64_t total_launches;
+    int32_t last_sweeps;
+};
+
+static int g_sm_count_cache[64];
+
+int qn_sm_count() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 1;
+    if (dev >= 0 && dev < 64 && g_sm_count_cache[dev] > 0) return g_sm_count_cache[dev];
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 1;
+    if (dev >= 0 && dev < 64) g_sm_count_cache[dev] = sms;
+    return sms;
+}
+
+extern "C" const char* qn_strerror(qn_status s) {
+    switch (s) {
+        case QN_OK: return "ok";
+        case QN_ERR_INVALID: return "invalid argument";
+        case QN_ERR_ALLOC: return "allocation failed";
+        case QN_ERR_CUDA: return "CUDA runtime error";
+        case QN_ERR_STATE: return "call not valid in this state";
+        case QN_ERR_NOT_CONVERGED: return "Jacobi sweep limit reached";
+        case QN_ERR_NONFINITE: return "non-finite Gram";
+    }
+    return "unknown status";
+}
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+inline bool finite_d(double x) { return isfinite(x); }
+
+inline void begin_call(qn_handle h, cudaStream_t st) {
+    h->last_launches = 0;
+    h->last_stream = st;
+}
+
+inline void end_call(qn_handle h) { h->total_launches += h->last_launches; }
+
+// Bring the result block to the host (waits for the stream) and hand j / sigma to the caller.
+qn_status fetch_result(qn_handle h, cudaStream_t st, int32_t* j_out, double* sigma_out) {
+    if (cudaMemcpyAsync(h->host_result, h->result, sizeof(qn_result_block), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return QN_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return QN_ERR_CUDA;
+    if (j_out) *j_out = h->host_result->j;
+    if (sigma_out) memcpy(sigma_out, h->host_result->sigma, sizeof(double) * h->m);
+    h->last_sweeps = h->host_result->sweeps;
+    return static_cast<qn_status>(h->host_result->status);
+}
+
+qn_status check_step_args(qn_handle h, double tau, double lambda, const void* theta_new) {
+    if (!h || !theta_new) return QN_ERR_INVALID;
+    if (!finite_d(tau) || !finite_d(lambda) || !(lambda > 0.0)) return QN_ERR_INVALID;
+    return QN_OK;
+}
+
+bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return a0 < b0 + nb && b0 < a0 + na;
+}
+
+// Gram partials -> solve -> combine on device buffers.
+qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, double lambda, void* theta_new,
+                   cudaStream_t st) {
+    int np = 0;
+    if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st, &h->last_launches) !=
+        cudaSuccess)
+        return QN_ERR_CUDA;
+    qn_solve_params p;
+    memset(&p, 0, sizeof(p));
+    p.m = h->m;
+    p.source = QN_SRC_PARTIALS;
+    p.partials = h->partials;
+    p.num_partials = np;
+    p.tau = tau;
+    p.lambda = lambda;
+    p.coef = h->coef;
+    p.result = h->result;
+    if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) return QN_ERR_CUDA;
+    if (qn_launch_combine(h->dtype, theta, g, h->n, h->m, h->coef, theta_new, st, &h->last_launches) != cudaSuccess)
+        return QN_ERR_CUDA;
+    return QN_OK;
+}
+
+qn_status ensure_window(qn_handle h) {
+    if (h->win_theta) return QN_OK;
+    const size_t bytes = (size_t)h->m * (size_t)h->n * h->elem;
+    void *a = nullptr, *b = nullptr;
+    if (cudaMalloc(&a, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return QN_ERR_ALLOC;
+    }
+    if (cudaMalloc(&b, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(a);
+        return QN_ERR_ALLOC;
+    }
+    h->win_theta = a;
+    h->win_g = b;
+    h->filled = 0;
+    h->head = 0;
+    return QN_OK;
+}
+
+}  // namespace
+
+extern "C" qn_status qn_create(int64_t n, int32_t m, qn_dtype dtype, qn_handle* out) {
+    if (!out || n < 1 || m < 1 || m > QN_MAX_M || (dtype != QN_F32 && dtype != QN_BF16)) return QN_ERR_INVALID;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        return QN_ERR_CUDA;
+    }
+    if (qn_solve_init() != cudaSuccess) {
+        cudaGetLastError();
+        return QN_ERR_CUDA;
+    }
+    qn_ctx* h = new (std::nothrow) qn_ctx();
+    if (!h) return QN_ERR_ALLOC;
+    memset(h, 0, sizeof(*h));
+    h->n = n;
+    h->m = m;
+    h->dtype = dtype;
+    h->elem = dtype == QN_F32 ? 4 : 2;
+    h->device = dev;
+    h->last_sweeps = -1;
+    h->max_partials = qn_sm_count() * 4;
+    bool ok = cudaMalloc(&h->partials, sizeof(double) * (size_t)h->max_partials * qn_partial_len(m)) == cudaSuccess;
+    ok = ok && cudaMalloc(&h->coef, sizeof(qn_coef_block)) == cudaSuccess;
+    ok = ok && cudaMalloc(&h->result, sizeof(qn_result_block)) == cudaSuccess;
+    ok = ok && cudaMalloc(&h->raw_gram, sizeof(double) * m * m) == cudaSuccess;
+    ok = ok && cudaMalloc(&h->ticket, sizeof(unsigned int)) == cudaSuccess;
+    ok = ok && cudaMallocHost(&h->host_result, sizeof(qn_result_block)) == cudaSuccess;
+    ok = ok && cudaMemset(h->ticket, 0, sizeof(unsigned int)) == cudaSuccess;
+    ok = ok && cudaMemset(h->result, 0, sizeof(qn_result_block)) == cudaSuccess;
+    ok = ok && cudaMemset(h->raw_gram, 0, sizeof(double) * m * m) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        qn_destroy(h);
+        return QN_ERR_ALLOC;
+    }
+    *out = h;
+    return QN_OK;
+}
+
+extern "C" qn_status qn_destroy(qn_handle h) {
+    if (!h) return QN_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    cudaDeviceSynchronize();
+    cudaFree(h->partials);
+    cudaFree(h->coef);
+    cudaFree(h->result);
+    cudaFree(h->raw_gram);
+    cudaFree(h->ticket);
+    cudaFree(h->win_theta);
+    cudaFree(h->win_g);
+    cudaFree(h->stage_theta);
+    cudaFree(h->stage_g);
+    cudaFree(h->stage_out);
+    if (h->host_result) cudaFreeHost(h->host_result);
+    cudaGetLastError();
+    delete h;
+    return QN_OK;
+}
+
+extern "C" qn_status qn_update(qn_handle h, const void* theta, const void* g, double tau, double lambda,
+                               void* theta_new, int32_t* j_out, double* sigma_out, void* cuda_stream) {
+    qn_status s = check_step_args(h, tau, lambda, theta_new);
+    if (s != QN_OK) return s;
+    if (!theta || !g) return QN_ERR_INVALID;
+    const size_t in_bytes = (size_t)h->m * (size_t)h->n * h->elem, out_bytes = (size_t)h->n * h->elem;
+    if (overlaps(theta_new, out_bytes, theta, in_bytes) || overlaps(theta_new, out_bytes, g, in_bytes))
+        return QN_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return QN_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    begin_call(h, st);
+    s = run_step(h, theta, g, tau, lambda, theta_new, st);
+    end_call(h);
+    if (s != QN_OK) return s;
+    if (j_out || sigma_out) return fetch_result(h, st, j_out, sigma_out);
+    return QN_OK;
+}
+
+extern "C" qn_status qn_gram(qn_handle h, const void* g, double* gram_out, void* cuda_stream) {
+    if (!h || !g || !gram_out) return QN_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return QN_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    begin_call(h, st);
+    int np = 0;
+    qn_status s = QN_OK;
+    if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st, &h->last_launches) !=
+        cudaSuccess)
+        s = QN_ERR_CUDA;
+    if (s == QN_OK) {
+        qn_solve_params p;
+        memset(&p, 0, sizeof(p));
+        p.m = h->m;
+        p.source = QN_SRC_PARTIALS;
+        p.partials = h->partials;
+        p.num_partials = np;
+        p.gram_out = gram_out;
+        p.gram_only = 1;
+        p.lambda = 1.0;
+        p.coef = h->coef;
+        p.result = h->result;
+        if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) s = QN_ERR_CUDA;
+    }
+    end_call(h);
+    return s;
+}
+
+extern "C" qn_status qn_window_alloc(qn_handle h) {
+    if (!h) return QN_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return QN_ERR_CUDA;
+    return ensure_window(h);
+}
+
+extern "C" void* qn_window_theta(qn_handle h) { return h ? h->win_theta : nullptr; }
+extern "C" void* qn_window_g(qn_handle h) { return h ? h->win_g : nullptr; }
+
+extern "C" qn_status qn_window_mark_full(qn_handle h) {
+    if (!h) return QN_ERR_INVALID;
+    if (!h->win_theta) return QN_ERR_STATE;
+    h->filled = h->m == 64 ? ~0ull : ((1ull << h->m) - 1ull);
+    return QN_OK;
+}
+
+extern "C" qn_status qn_push(qn_handle h, int32_t slot, const void* theta_col, const void* g_col, void* cuda_stream) {
+    if (!h || !theta_col || !g_col || slot < -1 || slot >= h->m) return QN_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return QN_ERR_CUDA;
+    qn_status s = ensure_window(h);
+    if (s != QN_OK) return s;
+    const size_t col_bytes = (size_t)h->n * h->elem, win_bytes = col_bytes * h->m;
+    if (overlaps(theta_col, col_bytes, h->win_theta, win_bytes) || overlaps(g_col, col_bytes, h->win_g, win_bytes))
+        return QN_ERR_INVALID;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    begin_call(h, st);
+    if (slot < 0) {
+        slot = h->head;
+        h->head = (h->head + 1) % h->m;
+    }
+    char* trow = static_cast<char*>(h->win_theta) + (size_t)slot * col_bytes;
+    char* grow = static_cast<char*>(h->win_g) + (size_t)slot * col_bytes;
+    if (cudaMemcpyAsync(trow, theta_col, col_bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess) s = QN_ERR_CUDA;
+    if (s == QN_OK && qn_launch_row(h->dtype, h->win_g, g_col, grow, h->n, h->m, slot, h->partials, h->max_partials,
+                                    h->raw_gram, h->ticket, st, &h->last_launches) != cudaSuccess)
+        s = QN_ERR_CUDA;
+    if (s == QN_OK) h->filled |= (1ull << slot);
+    end_call(h);
+    return s;
+}
+
+extern "C" qn_status qn_update_window(qn_handle h, double tau, double lambda, void* theta_new, int32_t* j_out,
+                                      double* sigma_out, void* cuda_stream) {
+    qn_status s = check_step_args(h, tau, lambda, theta_new);
+    if (s != QN_OK) return s;
+    const uint64_t full = h->m == 64 ? ~0ull : ((1ull << h->m) - 1ull);
+    if (!h->win_theta || h->filled != full) return QN_ERR_STATE;
+    const size_t win_bytes = (size_t)h->m * (size_t)h->n * h->elem, out_bytes = (size_t)h->n * h->elem;
+    if (overlaps(theta_new, out_bytes, h->win_theta, win_bytes) || overlaps(theta_new, out_bytes, h->win_g, win_bytes))
+        return QN_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return QN_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    begin_call(h, st);
+    qn_solve_params p;
+    memset(&p, 0, sizeof(p));
+    p.m = h->m;
+    p.source = QN_SRC_WINDOW;
+    p.raw_gram = h->raw_gram;
+    p.tau = tau;
+    p.lambda = lambda;
+    p.coef = h->coef;
+    p.result = h->result;
+    if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) s = QN_ERR_CUDA;
+    if (s == QN_OK && qn_launch_combine(h->dtype, h->win_theta, h->win_g, h->n, h->m, h->coef, theta_new, st,
+                                        &h->last_launches) != cudaSuccess)
+        s = QN_ERR_CUDA;
+    end_call(h);
+    if (s != QN_OK) return s;
+    if (j_out || sigma_out) return fetch_result(h, st, j_out, sigma_out);
+    return QN_OK;
+}
+
+extern "C" qn_status qn_rebuild(qn_handle h, void* cuda_stream) {
+    if (!h) return QN_ERR_INVALID;
+    if (!h->win_theta) return QN_ERR_STATE;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return QN_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    begin_call(h, st);
+    int np = 0;
+    qn_status s = QN_OK;
+    if (qn_launch_gram(h->dtype, h->win_g, h->n, h->m, true, h->partials, &np, h->max_partials, st,
+                       &h->last_launches) != cudaSuccess)
+        s = QN_ERR_CUDA;
+    if (s == QN_OK) {
+        qn_solve_params p;
+        memset(&p, 0, sizeof(p));
+        p.m = h->m;
+        p.source = QN_SRC_PARTIALS;
+        p.partials = h->partials;
+        p.num_partials = np;
+        p.raw_gram = h->raw_gram;
+        p.gram_only = 1;
+        p.lambda = 1.0;
+        p.coef = h->coef;
+        p.result = h->result;
+        if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) s = QN_ERR_CUDA;
+    }
+    end_call(h);
+    return s;
+}
+
+extern "C" qn_status qn_update_host(qn_handle h, const void* theta_host, const void* g_host, double tau, double lambda,
+                                    void* theta_new_host, int32_t* j_out, double* sigma_out, void* cuda_stream) {
+    qn_status s = check_step_args(h, tau, lambda, theta_new_host);
+    if (s != QN_OK) return s;
+    if (!theta_host || !g_host) return QN_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return QN_ERR_CUDA;
+    const size_t in_bytes = (size_t)h->m * (size_t)h->n * h->elem, out_bytes = (size_t)h->n * h->elem;
+    if (!h->stage_theta) {
+        bool ok = cudaMalloc(&h->stage_theta, in_bytes) == cudaSuccess;
+        ok = ok && cudaMalloc(&h->stage_g, in_bytes) == cudaSuccess;
+        ok = ok && cudaMalloc(&h->stage_out, out_bytes) == cudaSuccess;
+        if (!ok) {
+            cudaGetLastError();
+            cudaFree(h->stage_theta);
+            cudaFree(h->stage_g);
+            cudaFree(h->stage_out);
+            h->stage_theta = h->stage_g = h->stage_out = nullptr;
+            return QN_ERR_ALLOC;
+        }
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    begin_call(h, st);
+    // g first: the Gram pass needs only g, so theta's copy can overlap it on a copy engine
+    if (cudaMemcpyAsync(h->stage_g, g_host, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) s = QN_ERR_CUDA;
+    if (s == QN_OK && cudaMemcpyAsync(h->stage_theta, theta_host, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        s = QN_ERR_CUDA;
+    if (s == QN_OK) s = run_step(h, h->stage_theta, h->stage_g, tau, lambda, h->stage_out, st);
+    if (s == QN_OK &&
+        cudaMemcpyAsync(theta_new_host, h->stage_out, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        s = QN_ERR_CUDA;
+    end_call(h);
+    if (s != QN_OK) return s;
+    return fetch_result(h, st, j_out, sigma_out);
+}
+
+extern "C" qn_status qn_status_sync(qn_handle h) {
+    if (!h) return QN_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return QN_ERR_CUDA;
+    return fetch_result(h, h->last_stream, nullptr, nullptr);
+}
+
+extern "C" int32_t qn_last_launches(qn_handle h) { return h ? h->last_launches : 0; }
+extern "C" int64_t qn_total_launches(qn_handle h) { return h ? h->total_launches : 0; }
+extern "C" int32_t qn_last_sweeps(qn_handle h) { return h ? h->last_sweeps : -1; }

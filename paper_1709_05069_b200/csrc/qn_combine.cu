@@ -1,0 +1,134 @@
+// Final streaming pass: theta_new = thetabar - tau*(gbar - G d + Theta d)  (paper, Eq. (2) with the
+// operator of Eq. (4) applied to gbar; G d and Theta d are the two sums of Eq. (4) collapsed onto the
+// m-vector d built by the solve kernel).  With c = tau*(d - mean(d)), sum(c) = 0 and
+//     theta_new[i] = mean_k theta[k][i] - tau * mean_k g[k][i]
+//                    + sum_k c[k] * ((g[k][i] - g[0][i]) - (theta[k][i] - theta[0][i])).
+// Differences against Worker 0 are formed before the multiplication so that the rounding of each
+// term is relative to the Workers' spread, not to the magnitude of theta and g.  fp32 arithmetic,
+// fixed summation order k = 0..m-1, one rounding to the storage type.  Neither the means nor the
+// centred matrices are ever stored: the pass reads 2*m*n elements and writes n.
+#include "qn_device.cuh"
+
+namespace qn {
+
+constexpr int kCombineThreads = 256;
+constexpr int kCombineUnroll = 4;  // Workers whose loads are in flight together
+
+template <typename T, bool kAligned>
+__global__ void __launch_bounds__(kCombineThreads)
+combine_kernel(const T* __restrict__ theta, const T* __restrict__ g, int64_t n, int m,
+               const qn_coef_block* __restrict__ coef, T* __restrict__ out) {
+    constexpr int kCols = kAligned ? Storage<T>::kVec : 1;
+    __shared__ float c_sh[QN_MAX_M];
+    if (threadIdx.x < QN_MAX_M) c_sh[threadIdx.x] = coef->c[threadIdx.x];
+    const float tau = coef->tau, inv_m = coef->inv_m;
+    __syncthreads();
+
+    const int64_t nitems = kAligned ? n / kCols : n;
+    for (int64_t item = (int64_t)blockIdx.x * kCombineThreads + threadIdx.x; item < nitems;
+         item += (int64_t)gridDim.x * kCombineThreads) {
+        const int64_t i0 = item * kCols;
+        float th0[kCols], g0[kCols], sth[kCols], sg[kCols], acc[kCols];
+        {
+            uint4 a, b;
+            if (kAligned) {
+                a = ldg_stream16(theta + i0);
+                b = ldg_stream16(g + i0);
+            } else {
+                a.x = __float_as_uint(Storage<T>::load1(theta + i0));
+                b.x = __float_as_uint(Storage<T>::load1(g + i0));
+            }
+#pragma unroll
+            for (int e = 0; e < kCols; ++e) {
+                th0[e] = kAligned ? Storage<T>::get(a, e) : __uint_as_float(a.x);
+                g0[e] = kAligned ? Storage<T>::get(b, e) : __uint_as_float(b.x);
+                sth[e] = th0[e];
+                sg[e] = g0[e];
+                acc[e] = 0.f;
+            }
+        }
+        int k = 1;
+        for (; k + kCombineUnroll <= m; k += kCombineUnroll) {
+            uint4 a[kCombineUnroll], b[kCombineUnroll];
+#pragma unroll
+            for (int u = 0; u < kCombineUnroll; ++u) {
+                if (kAligned) {
+                    a[u] = ldg_stream16(theta + (int64_t)(k + u) * n + i0);
+                    b[u] = ldg_stream16(g + (int64_t)(k + u) * n + i0);
+                } else {
+                    a[u].x = __float_as_uint(Storage<T>::load1(theta + (int64_t)(k + u) * n + i0));
+                    b[u].x = __float_as_uint(Storage<T>::load1(g + (int64_t)(k + u) * n + i0));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kCombineUnroll; ++u) {
+                const float ck = c_sh[k + u];
+#pragma unroll
+                for (int e = 0; e < kCols; ++e) {
+                    const float t = kAligned ? Storage<T>::get(a[u], e) : __uint_as_float(a[u].x);
+                    const float gg = kAligned ? Storage<T>::get(b[u], e) : __uint_as_float(b[u].x);
+                    sth[e] += t;
+                    sg[e] += gg;
+                    acc[e] = fmaf(ck, (gg - g0[e]) - (t - th0[e]), acc[e]);
+                }
+            }
+        }
+        for (; k < m; ++k) {
+            uint4 a, b;
+            if (kAligned) {
+                a = ldg_stream16(theta + (int64_t)k * n + i0);
+                b = ldg_stream16(g + (int64_t)k * n + i0);
+            } else {
+                a.x = __float_as_uint(Storage<T>::load1(theta + (int64_t)k * n + i0));
+                b.x = __float_as_uint(Storage<T>::load1(g + (int64_t)k * n + i0));
+            }
+            const float ck = c_sh[k];
+#pragma unroll
+            for (int e = 0; e < kCols; ++e) {
+                const float t = kAligned ? Storage<T>::get(a, e) : __uint_as_float(a.x);
+                const float gg = kAligned ? Storage<T>::get(b, e) : __uint_as_float(b.x);
+                sth[e] += t;
+                sg[e] += gg;
+                acc[e] = fmaf(ck, (gg - g0[e]) - (t - th0[e]), acc[e]);
+            }
+        }
+        float res[kCols];
+#pragma unroll
+        for (int e = 0; e < kCols; ++e) res[e] = fmaf(-tau * inv_m, sg[e], fmaf(sth[e], inv_m, acc[e]));
+        if (kAligned) {
+            stg_stream16(out + i0, Storage<T>::pack(res));
+        } else {
+            Storage<T>::store1(out + i0, res[0]);
+        }
+    }
+}
+
+template <typename T>
+static cudaError_t launch_combine_t(const T* theta, const T* g, int64_t n, int m, const qn_coef_block* coef, T* out,
+                                    cudaStream_t st) {
+    const bool aligned = (reinterpret_cast<uintptr_t>(theta) % 16 == 0) && (reinterpret_cast<uintptr_t>(g) % 16 == 0) &&
+                         (reinterpret_cast<uintptr_t>(out) % 16 == 0) && ((n * (int64_t)sizeof(T)) % 16 == 0);
+    const int64_t nitems = aligned ? n / Storage<T>::kVec : n;
+    const int64_t want = (nitems + kCombineThreads - 1) / kCombineThreads;
+    const int64_t cap = (int64_t)qn_sm_count() * 8;
+    const int grid = (int)(want < cap ? (want > 0 ? want : 1) : cap);
+    if (aligned)
+        combine_kernel<T, true><<<grid, kCombineThreads, 0, st>>>(theta, g, n, m, coef, out);
+    else
+        combine_kernel<T, false><<<grid, kCombineThreads, 0, st>>>(theta, g, n, m, coef, out);
+    return cudaGetLastError();
+}
+
+}  // namespace qn
+
+cudaError_t qn_launch_combine(qn_dtype dtype, const void* theta, const void* g, int64_t n, int m,
+                              const qn_coef_block* coef, void* theta_new, cudaStream_t st, int* launches) {
+    cudaError_t e =
+        dtype == QN_F32
+            ? qn::launch_combine_t(static_cast<const float*>(theta), static_cast<const float*>(g), n, m, coef,
+                                   static_cast<float*>(theta_new), st)
+            : qn::launch_combine_t(static_cast<const __nv_bfloat16*>(theta), static_cast<const __nv_bfloat16*>(g), n, m,
+                                   coef, static_cast<__nv_bfloat16*>(theta_new), st);
+    if (e == cudaSuccess && launches) *launches += 1;
+    return e;
+}

@@ -1,0 +1,69 @@
+// Device helpers: streaming 128-bit loads, storage-type unpacking, block reductions.
+#pragma once
+
+#include "qn_internal.h"
+
+namespace qn {
+
+template <typename T>
+struct Storage;
+
+template <>
+struct Storage<float> {
+    static constexpr int kVec = 4;  // elements per 16-byte vector
+    __device__ static __forceinline__ float get(const uint4& v, int e) {
+        const uint32_t w = e == 0 ? v.x : e == 1 ? v.y : e == 2 ? v.z : v.w;
+        return __uint_as_float(w);
+    }
+    __device__ static __forceinline__ float load1(const float* p) { return __ldg(p); }
+    __device__ static __forceinline__ void store1(float* p, float x) { *p = x; }
+    __device__ static __forceinline__ uint4 pack(const float* x) {
+        return make_uint4(__float_as_uint(x[0]), __float_as_uint(x[1]), __float_as_uint(x[2]), __float_as_uint(x[3]));
+    }
+};
+
+template <>
+struct Storage<__nv_bfloat16> {
+    static constexpr int kVec = 8;
+    __device__ static __forceinline__ float get(const uint4& v, int e) {
+        const uint32_t w = (e >> 1) == 0 ? v.x : (e >> 1) == 1 ? v.y : (e >> 1) == 2 ? v.z : v.w;
+        return __uint_as_float((e & 1) ? (w & 0xffff0000u) : (w << 16));
+    }
+    __device__ static __forceinline__ float load1(const __nv_bfloat16* p) {
+        return __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(p))) << 16);
+    }
+    __device__ static __forceinline__ void store1(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+    __device__ static __forceinline__ uint4 pack(const float* x) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            // cvt.rn.bf16x2.f32 d, a, b: a -> upper half, b -> lower half
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(x[2 * i + 1]), "f"(x[2 * i]));
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+// 16-byte read-only load that does not allocate in L1 (every input element is read once per pass).
+__device__ __forceinline__ uint4 ldg_stream16(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// 16-byte streaming store (written once, not re-read by this kernel).
+__device__ __forceinline__ void stg_stream16(void* p, const uint4& v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+// Sum over the warp in a fixed butterfly order; every lane ends with the same value.
+__device__ __forceinline__ double warp_sum(double x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+}  // namespace qn

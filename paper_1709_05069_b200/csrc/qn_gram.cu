@@ -1,0 +1,371 @@
+// Streaming reduction over g[m][n]: per-column reference (the Workers' mean), shifted values
+// x_k = g_k - r, the Gram sum_i x_k x_l and the products t_k = sum_i x_k r, as per-CTA fp64 partials
+// in the packed layout of qn_internal.h.  (Section 2 of the paper: means, centred matrix G, G^H G
+// and the numerators of alpha_k for z = gbar.)  The solve kernel sums the partials in a fixed
+// order and applies the exact m x m centring, so any rounding in the per-column reference cancels.
+//
+// Arithmetic: fp32 products, fp32 accumulation over at most kFlushCols columns per thread, then
+// fp64.  Every thread owns fixed columns and fixed output entries, so results are bitwise
+// reproducible for a given grid.
+#include "qn_device.cuh"
+
+namespace qn {
+
+constexpr int kThreads = 256;
+constexpr int kFlushCols = 32;  // columns accumulated in fp32 by one thread between fp64 flushes
+
+// ------------------------------------------------------------------------------------------------
+// Direct kernel, m <= 8: one thread holds all m values of its columns in registers and owns a full
+// private copy of the 36 + 8 accumulators.
+// ------------------------------------------------------------------------------------------------
+constexpr int kDirectM = 8;
+constexpr int kDirectTri = kDirectM * (kDirectM + 1) / 2;  // 36
+constexpr int kDirectAcc = kDirectTri + kDirectM;          // 44
+
+template <typename T, bool kAligned>
+struct DirectItem {
+    // one work item = 16 bytes of every row (aligned) or one element of every row (unaligned)
+    static constexpr int kCols = kAligned ? Storage<T>::kVec : 1;
+    uint4 v[kDirectM];
+
+    __device__ __forceinline__ void load(const T* g, int64_t n, int m, int64_t item, int64_t nitems) {
+#pragma unroll
+        for (int k = 0; k < kDirectM; ++k) {
+            v[k] = make_uint4(0, 0, 0, 0);
+            if (k < m && item < nitems) {
+                if (kAligned) {
+                    v[k] = ldg_stream16(g + (int64_t)k * n + item * kCols);
+                } else {
+                    v[k].x = __float_as_uint(Storage<T>::load1(g + (int64_t)k * n + item));
+                }
+            }
+        }
+    }
+    __device__ __forceinline__ float get(int k, int e) const {
+        return kAligned ? Storage<T>::get(v[k], e) : __uint_as_float(v[k].x);
+    }
+};
+
+template <typename T, bool kAligned, bool kRaw>
+__global__ void __launch_bounds__(kThreads, 1)
+gram_direct_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ partials) {
+    using Item = DirectItem<T, kAligned>;
+    constexpr int kCols = Item::kCols;
+    constexpr int kFlushIters = kFlushCols / kCols > 0 ? kFlushCols / kCols : 1;
+
+    const int64_t nitems = kAligned ? n / kCols : n;
+    const int64_t ntiles = (nitems + kThreads - 1) / kThreads;
+
+    float acc[kDirectAcc];
+    double acc64[kDirectAcc];
+#pragma unroll
+    for (int e = 0; e < kDirectAcc; ++e) {
+        acc[e] = 0.f;
+        acc64[e] = 0.0;
+    }
+    float mask[kDirectM];  // 1 for real Workers, 0 for the padding rows
+#pragma unroll
+    for (int k = 0; k < kDirectM; ++k) mask[k] = k < m ? 1.f : 0.f;
+    const float inv_m = 1.0f / (float)m;
+
+    Item cur, nxt;
+    int64_t tile = blockIdx.x;
+    cur.load(g, n, m, tile * kThreads + threadIdx.x, tile < ntiles ? nitems : 0);
+    int iters = 0;
+    for (; tile < ntiles; tile += gridDim.x) {
+        const int64_t next_tile = tile + gridDim.x;
+        nxt.load(g, n, m, next_tile * kThreads + threadIdx.x, next_tile < ntiles ? nitems : 0);
+#pragma unroll
+        for (int e = 0; e < kCols; ++e) {
+            float x[kDirectM];
+            float s = 0.f;
+#pragma unroll
+            for (int k = 0; k < kDirectM; ++k) {
+                x[k] = cur.get(k, e);
+                s += x[k];
+            }
+            if (kRaw) {
+                // raw Gram (reference 0), accumulated directly in fp64: products of fp32 or bf16
+                // values are exact in fp64
+#pragma unroll
+                for (int k = 0, idx = 0; k < kDirectM; ++k) {
+                    const double xk = (double)x[k];
+#pragma unroll
+                    for (int l = k; l < kDirectM; ++l, ++idx) acc64[idx] = fma(xk, (double)x[l], acc64[idx]);
+                }
+            } else {
+                const float r = s * inv_m;
+#pragma unroll
+                for (int k = 0; k < kDirectM; ++k) x[k] = fmaf(-mask[k], r, x[k]);
+#pragma unroll
+                for (int k = 0, idx = 0; k < kDirectM; ++k) {
+#pragma unroll
+                    for (int l = k; l < kDirectM; ++l, ++idx) acc[idx] = fmaf(x[k], x[l], acc[idx]);
+                }
+#pragma unroll
+                for (int k = 0; k < kDirectM; ++k) acc[kDirectTri + k] = fmaf(x[k], r, acc[kDirectTri + k]);
+            }
+        }
+        if (!kRaw && ++iters == kFlushIters) {
+            iters = 0;
+#pragma unroll
+            for (int e = 0; e < kDirectAcc; ++e) {
+                acc64[e] += (double)acc[e];
+                acc[e] = 0.f;
+            }
+        }
+        cur = nxt;
+    }
+    if (!kRaw) {
+#pragma unroll
+        for (int e = 0; e < kDirectAcc; ++e) acc64[e] += (double)acc[e];
+    }
+
+    // CTA reduction in a fixed order: butterfly inside each warp, then warps 0..7 in sequence.
+    __shared__ double red[kThreads / 32][kDirectAcc];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int e = 0; e < kDirectAcc; ++e) {
+        const double s = warp_sum(acc64[e]);
+        if (lane == 0) red[warp][e] = s;
+    }
+    __syncthreads();
+    if (threadIdx.x < kDirectAcc) {
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) s += red[w][threadIdx.x];
+        // map the 8-row packed index to the m-row packed index
+        const int e = threadIdx.x;
+        double* out = partials + (int64_t)blockIdx.x * qn_partial_len(m);
+        if (e < kDirectTri) {
+            int k = 0, rem = e;
+            while (rem >= kDirectM - k) {
+                rem -= kDirectM - k;
+                ++k;
+            }
+            const int l = k + rem;
+            if (l < m) out[qn_tri_index(m, k, l)] = s;
+        } else {
+            const int k = e - kDirectTri;
+            if (k < m) out[m * (m + 1) / 2 + k] = s;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Tiled kernel, 9 <= m <= 64, plain fp32 ALUs.  A tile of kTileCols columns is staged in shared
+// memory as shifted fp32 values, one record of RBP floats per column: rows 0..m-1 = x_k, row m =
+// the reference r (so that entry (k, m) of the extended Gram is t_k), zero padding up to a
+// multiple of 8.  The extended Gram is cut into 8x8 blocks; a thread owns one upper-triangle block
+// and a fixed residue class of the tile's columns, with the 64 accumulators in registers.
+// ------------------------------------------------------------------------------------------------
+constexpr int kTileCols = 128;
+constexpr int kMaxBlocks = (QN_MAX_M + 1 + 7) / 8;                 // 9
+constexpr int kMaxRBP = 8 * kMaxBlocks + 4;                        // 76 floats per column record
+
+struct TiledSmem {
+    float xs[kTileCols * kMaxRBP];
+    float psum[kTileCols * 17];
+};
+
+template <typename T, bool kAligned, bool kRaw>
+__global__ void __launch_bounds__(kThreads, 1)
+gram_tiled_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ partials) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    TiledSmem& sm = *reinterpret_cast<TiledSmem*>(smem_raw);
+
+    constexpr int kCols = kAligned ? Storage<T>::kVec : 1;  // columns per load item
+    constexpr int kColGroups = kTileCols / kCols;           // load items per row per tile
+    constexpr int kRowGroups = kThreads / kColGroups;       // 8 (fp32 x4), 16 (bf16 x8), 2 (scalar)
+
+    const int nb = (m + 1 + 7) / 8;
+    const int RB = 8 * nb;
+    const int RBP = RB + 4;
+    const int ntile = nb * (nb + 1) / 2;
+    int S = 8;
+    while (S < ntile) S <<= 1;  // slots per column step: 8, 16, 32 or 64
+    const int slot = threadIdx.x % S;
+    const int col0 = threadIdx.x / S;
+    const int colstep = kThreads / S;
+    const bool active = slot < ntile;
+
+    __shared__ unsigned char tile_a[64], tile_b[64];  // block coordinates of each slot
+    if (threadIdx.x < 64) {
+        int t = 0;
+        for (int a = 0; a < nb; ++a)
+            for (int b = a; b < nb; ++b, ++t)
+                if (t == (int)threadIdx.x) {
+                    tile_a[t] = (unsigned char)a;
+                    tile_b[t] = (unsigned char)b;
+                }
+    }
+    __syncthreads();
+    const int ta = active ? tile_a[slot] : 0, tb = active ? tile_b[slot] : 0;
+
+    float acc[64];
+    double acc64[64];
+#pragma unroll
+    for (int e = 0; e < 64; ++e) {
+        acc[e] = 0.f;
+        acc64[e] = 0.0;
+    }
+    const float inv_m = 1.0f / (float)m;
+    const int rg = threadIdx.x % kRowGroups, cg = threadIdx.x / kRowGroups;
+    const int64_t ntiles = (n + kTileCols - 1) / kTileCols;
+    int cols_since_flush = 0;
+
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const int64_t i0 = tile * kTileCols + (int64_t)cg * kCols;
+        // pass A: raw values into the column records, partial sums over this thread's rows
+        float ps[kCols];
+#pragma unroll
+        for (int e = 0; e < kCols; ++e) ps[e] = 0.f;
+        for (int k = rg; k < m; k += kRowGroups) {
+            float val[kCols];
+            if (kAligned) {
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (i0 < n) v = ldg_stream16(g + (int64_t)k * n + i0);
+#pragma unroll
+                for (int e = 0; e < kCols; ++e) val[e] = Storage<T>::get(v, e);
+            } else {
+                val[0] = i0 < n ? Storage<T>::load1(g + (int64_t)k * n + i0) : 0.f;
+            }
+#pragma unroll
+            for (int e = 0; e < kCols; ++e) {
+                sm.xs[(cg * kCols + e) * RBP + k] = val[e];
+                ps[e] += val[e];
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < kCols; ++e) sm.psum[(cg * kCols + e) * (kRowGroups + 1) + rg] = ps[e];
+        __syncthreads();
+        // pass B: reference of this thread's columns (fixed summation order), shift own entries
+        float r[kCols];
+#pragma unroll
+        for (int e = 0; e < kCols; ++e) {
+            float s = 0.f;
+            for (int q = 0; q < kRowGroups; ++q) s += sm.psum[(cg * kCols + e) * (kRowGroups + 1) + q];
+            r[e] = kRaw ? 0.f : s * inv_m;
+        }
+        if (!kRaw) {
+            for (int k = rg; k < m; k += kRowGroups) {
+#pragma unroll
+                for (int e = 0; e < kCols; ++e) sm.xs[(cg * kCols + e) * RBP + k] -= r[e];
+            }
+        }
+        if (rg == 0) {
+#pragma unroll
+            for (int e = 0; e < kCols; ++e) {
+                sm.xs[(cg * kCols + e) * RBP + m] = r[e];
+                for (int k = m + 1; k < RB; ++k) sm.xs[(cg * kCols + e) * RBP + k] = 0.f;
+            }
+        }
+        __syncthreads();
+        // compute: this thread's 8x8 block over its residue class of columns
+        if (active) {
+            for (int c = col0; c < kTileCols; c += colstep) {
+                const float4* rec = reinterpret_cast<const float4*>(&sm.xs[c * RBP]);
+                const float4 a0 = rec[2 * ta], a1 = rec[2 * ta + 1];
+                const float4 b0 = rec[2 * tb], b1 = rec[2 * tb + 1];
+                const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+                const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+                for (int p = 0; p < 8; ++p)
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) acc[p * 8 + q] = fmaf(a[p], b[q], acc[p * 8 + q]);
+            }
+        }
+        cols_since_flush += kTileCols / colstep;
+        if (kRaw || cols_since_flush >= kFlushCols) {
+            cols_since_flush = 0;
+#pragma unroll
+            for (int e = 0; e < 64; ++e) {
+                acc64[e] += (double)acc[e];
+                acc[e] = 0.f;
+            }
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int e = 0; e < 64; ++e) acc64[e] += (double)acc[e];
+
+    // CTA reduction: for each block, sum the kThreads/S column classes in the order 0,1,2,...
+    double* red = reinterpret_cast<double*>(smem_raw);  // reuse of the tile storage: kThreads*16 doubles
+    double* out = partials + (int64_t)blockIdx.x * qn_partial_len(m);
+    const int tri_len = m * (m + 1) / 2;
+#pragma unroll
+    for (int part = 0; part < 4; ++part) {
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < 16; ++e) red[threadIdx.x * 16 + e] = acc64[part * 16 + e];
+        __syncthreads();
+        for (int w = threadIdx.x; w < S * 16; w += kThreads) {
+            const int sl = w / 16, e = part * 16 + (w % 16);
+            if (sl >= ntile) continue;
+            double s = 0.0;
+            for (int q = 0; q < colstep; ++q) s += red[(q * S + sl) * 16 + (w % 16)];
+            const int row = 8 * tile_a[sl] + e / 8, col = 8 * tile_b[sl] + e % 8;
+            if (row < m && row <= col) {
+                if (col < m)
+                    out[qn_tri_index(m, row, col)] = s;
+                else if (col == m)
+                    out[tri_len + row] = s;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+static cudaError_t launch_gram_t(const T* g, int64_t n, int m, bool raw, double* partials, int* num_partials,
+                                 int max_partials, cudaStream_t st) {
+    const bool aligned = (reinterpret_cast<uintptr_t>(g) % 16 == 0) && ((n * (int64_t)sizeof(T)) % 16 == 0);
+    const int sms = qn_sm_count();
+    if (m <= kDirectM) {
+        const int64_t nitems = aligned ? n / Storage<T>::kVec : n;
+        const int64_t ntiles = (nitems + kThreads - 1) / kThreads;
+        int grid = (int)(ntiles < sms ? ntiles : sms);
+        if (grid > max_partials) grid = max_partials;
+        *num_partials = grid;
+        if (aligned) {
+            if (raw)
+                gram_direct_kernel<T, true, true><<<grid, kThreads, 0, st>>>(g, n, m, partials);
+            else
+                gram_direct_kernel<T, true, false><<<grid, kThreads, 0, st>>>(g, n, m, partials);
+        } else {
+            if (raw)
+                gram_direct_kernel<T, false, true><<<grid, kThreads, 0, st>>>(g, n, m, partials);
+            else
+                gram_direct_kernel<T, false, false><<<grid, kThreads, 0, st>>>(g, n, m, partials);
+        }
+        return cudaGetLastError();
+    }
+    const int64_t ntiles = (n + kTileCols - 1) / kTileCols;
+    int grid = (int)(ntiles < sms ? ntiles : sms);
+    if (grid > max_partials) grid = max_partials;
+    *num_partials = grid;
+    const size_t smem = sizeof(TiledSmem);
+    auto go = [&](auto kern) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<grid, kThreads, smem, st>>>(g, n, m, partials);
+        return cudaGetLastError();
+    };
+    if (aligned) return raw ? go(gram_tiled_kernel<T, true, true>) : go(gram_tiled_kernel<T, true, false>);
+    return raw ? go(gram_tiled_kernel<T, false, true>) : go(gram_tiled_kernel<T, false, false>);
+}
+
+}  // namespace qn
+
+cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
+                           int* num_partials, int max_partials, cudaStream_t st, int* launches) {
+    cudaError_t e = dtype == QN_F32
+                        ? qn::launch_gram_t(static_cast<const float*>(g), n, m, raw, partials, num_partials,
+                                            max_partials, st)
+                        : qn::launch_gram_t(static_cast<const __nv_bfloat16*>(g), n, m, raw, partials, num_partials,
+                                            max_partials, st);
+    if (e == cudaSuccess && launches) *launches += 1;
+    return e;
+}

@@ -1,0 +1,65 @@
+// Internal declarations shared by the .cu files of libqn (not part of the public ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "qn.h"
+
+// Packed layout of one Gram partial for m Workers: the upper triangle of the (reference-shifted)
+// Gram by rows, entry (k,l), k <= l, at k*m - k*(k-1)/2 + (l-k), followed by t[m] (the products of
+// each shifted row with the per-column reference).
+__host__ __device__ inline int qn_tri_index(int m, int k, int l) { return k * m - (k * (k - 1)) / 2 + (l - k); }
+__host__ __device__ inline int qn_partial_len(int m) { return m * (m + 1) / 2 + m; }
+
+// Device block read back by the host after a step.
+struct qn_result_block {
+    int32_t j;
+    int32_t status;  // qn_status seen on the device (OK, NOT_CONVERGED, NONFINITE)
+    int32_t sweeps;
+    int32_t pad;
+    double sigma[QN_MAX_M];
+};
+
+// Coefficients consumed by the combine kernel:
+// theta_new = mean(theta) - tau*mean(g) + sum_k c[k]*((g_k - g_0) - (theta_k - theta_0)).
+struct qn_coef_block {
+    float c[QN_MAX_M];
+    float tau;
+    float inv_m;
+    int32_t m;
+    int32_t pad;
+};
+
+// What the solve kernel starts from.
+enum qn_solve_source {
+    QN_SRC_PARTIALS = 0,  // sum `num_partials` packed partials; if raw_gram != NULL also store the sum there
+    QN_SRC_WINDOW = 1     // start from the raw Gram kept in `raw_gram` (reference 0, t = 0)
+};
+
+struct qn_solve_params {
+    int32_t m;
+    int32_t source;
+    const double* partials;  // [num_partials][qn_partial_len(m)]
+    int32_t num_partials;
+    double* raw_gram;     // m*m doubles: read (QN_SRC_WINDOW) or written with the uncentred sum (QN_SRC_PARTIALS)
+    double* gram_out;     // m*m + m doubles: centred C then w (may be NULL)
+    int32_t gram_only;    // stop after writing gram_out
+    double tau, lambda;
+    qn_coef_block* coef;
+    qn_result_block* result;
+};
+
+// Launchers.  Each returns the launch error and adds the kernels it launched to *launches.
+cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
+                           int* num_partials, int max_partials, cudaStream_t st, int* launches);
+cudaError_t qn_launch_solve(const qn_solve_params& p, cudaStream_t st, int* launches);
+cudaError_t qn_launch_combine(qn_dtype dtype, const void* theta, const void* g, int64_t n, int m,
+                              const qn_coef_block* coef, void* theta_new, cudaStream_t st, int* launches);
+cudaError_t qn_launch_row(qn_dtype dtype, const void* window_g, const void* g_col, void* window_row_out, int64_t n,
+                          int m, int slot, double* partials, int max_partials, double* raw_gram, unsigned int* ticket,
+                          cudaStream_t st, int* launches);
+cudaError_t qn_solve_init();
+
+int qn_sm_count();

@@ -1,0 +1,149 @@
+// Asynchronous mode: one Worker's Write replaces column `slot` of the window.  This pass lands the new
+// gradient column in the window and computes the one row of the window's RAW Gram that changed,
+// S[slot][l] = sum_i gnew[i] * g_l[i] for l = 0..m-1 (with g_slot = gnew), reading m*n elements
+// instead of the m*(m+1)/2 dot products of a full recomputation.  (The paper, Section 2, allows an
+// update after each Write but does not say what the Server keeps; the window and its raw Gram are
+// this library's reading.)
+//
+// The raw Gram has to carry the cancellation of the later m x m centring, so every product is
+// formed and accumulated in fp64 (products of two fp32 or bf16 values are exact in fp64).
+// The last CTA to finish adds the per-CTA partial rows in a fixed order and patches row and column
+// `slot` of the Gram: no CTA ever waits for another.
+#include "qn_device.cuh"
+
+namespace qn {
+
+constexpr int kRowThreads = 256;
+constexpr int kRowBlock = 8;  // window columns handled by one CTA row (blockIdx.y)
+
+template <typename T, bool kAligned>
+__global__ void __launch_bounds__(kRowThreads)
+row_kernel(const T* __restrict__ window_g, const T* __restrict__ g_col, T* __restrict__ window_row_out, int64_t n,
+           int m, int slot, double* __restrict__ partials, double* __restrict__ raw_gram, unsigned int* ticket) {
+    constexpr int kCols = kAligned ? Storage<T>::kVec : 1;
+    const int lb = blockIdx.y * kRowBlock;
+    const int64_t nitems = kAligned ? n / kCols : n;
+
+    double acc[kRowBlock];
+#pragma unroll
+    for (int r = 0; r < kRowBlock; ++r) acc[r] = 0.0;
+
+    for (int64_t item = (int64_t)blockIdx.x * kRowThreads + threadIdx.x; item < nitems;
+         item += (int64_t)gridDim.x * kRowThreads) {
+        const int64_t i0 = item * kCols;
+        uint4 xn, xl[kRowBlock];
+        if (kAligned)
+            xn = ldg_stream16(g_col + i0);
+        else
+            xn.x = __float_as_uint(Storage<T>::load1(g_col + i0));
+#pragma unroll
+        for (int r = 0; r < kRowBlock; ++r) {
+            const int l = lb + r;
+            xl[r] = make_uint4(0, 0, 0, 0);
+            if (l < m) {
+                if (l == slot)
+                    xl[r] = xn;
+                else if (kAligned)
+                    xl[r] = ldg_stream16(window_g + (int64_t)l * n + i0);
+                else
+                    xl[r].x = __float_as_uint(Storage<T>::load1(window_g + (int64_t)l * n + i0));
+            }
+        }
+        if (blockIdx.y == 0) {  // land the column
+            if (kAligned)
+                stg_stream16(window_row_out + i0, xn);
+            else
+                window_row_out[i0] = g_col[i0];
+        }
+#pragma unroll
+        for (int e = 0; e < kCols; ++e) {
+            const double a = (double)(kAligned ? Storage<T>::get(xn, e) : __uint_as_float(xn.x));
+#pragma unroll
+            for (int r = 0; r < kRowBlock; ++r) {
+                const double b = (double)(kAligned ? Storage<T>::get(xl[r], e) : __uint_as_float(xl[r].x));
+                acc[r] = fma(a, b, acc[r]);
+            }
+        }
+    }
+
+    __shared__ double red[kRowThreads / 32][kRowBlock];
+    __shared__ bool is_last;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int r = 0; r < kRowBlock; ++r) {
+        const double s = warp_sum(acc[r]);
+        if (lane == 0) red[warp][r] = s;
+    }
+    __syncthreads();
+    if (threadIdx.x < kRowBlock && lb + threadIdx.x < m) {
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < kRowThreads / 32; ++w) s += red[w][threadIdx.x];
+        partials[(int64_t)blockIdx.x * m + lb + threadIdx.x] = s;
+    }
+    // last-CTA-done: publish the partial, take a ticket; the CTA that draws the last ticket reduces
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int total = gridDim.x * gridDim.y;
+        const unsigned int t = atomicAdd(ticket, 1u);
+        is_last = (t == total - 1);
+    }
+    __syncthreads();
+    if (is_last) {
+        __threadfence();
+        if (threadIdx.x < m) {
+            double s0 = 0.0, s1 = 0.0;
+            unsigned int p = 0;
+            for (; p + 1 < gridDim.x; p += 2) {
+                s0 += __ldcg(&partials[(int64_t)p * m + threadIdx.x]);
+                s1 += __ldcg(&partials[(int64_t)(p + 1) * m + threadIdx.x]);
+            }
+            if (p < gridDim.x) s0 += __ldcg(&partials[(int64_t)p * m + threadIdx.x]);
+            const double v = s0 + s1;
+            raw_gram[slot * m + threadIdx.x] = v;
+            raw_gram[threadIdx.x * m + slot] = v;
+        }
+        if (threadIdx.x == 0) *ticket = 0;  // ready for the next launch on this stream
+    }
+}
+
+template <typename T>
+static cudaError_t launch_row_t(const T* window_g, const T* g_col, T* window_row_out, int64_t n, int m, int slot,
+                                double* partials, int max_partials, double* raw_gram, unsigned int* ticket,
+                                cudaStream_t st) {
+    const bool aligned = (reinterpret_cast<uintptr_t>(window_g) % 16 == 0) &&
+                         (reinterpret_cast<uintptr_t>(g_col) % 16 == 0) && ((n * (int64_t)sizeof(T)) % 16 == 0);
+    const int64_t nitems = aligned ? n / Storage<T>::kVec : n;
+    const int nby = (m + kRowBlock - 1) / kRowBlock;
+    int64_t want = (nitems + kRowThreads - 1) / kRowThreads;
+    int64_t cap = (int64_t)qn_sm_count() * 4 / nby;
+    if (cap < 1) cap = 1;
+    if (cap > max_partials) cap = max_partials;
+    const int gx = (int)(want < cap ? (want > 0 ? want : 1) : cap);
+    dim3 grid(gx, nby);
+    if (aligned)
+        row_kernel<T, true><<<grid, kRowThreads, 0, st>>>(window_g, g_col, window_row_out, n, m, slot, partials,
+                                                         raw_gram, ticket);
+    else
+        row_kernel<T, false><<<grid, kRowThreads, 0, st>>>(window_g, g_col, window_row_out, n, m, slot, partials,
+                                                          raw_gram, ticket);
+    return cudaGetLastError();
+}
+
+}  // namespace qn
+
+cudaError_t qn_launch_row(qn_dtype dtype, const void* window_g, const void* g_col, void* window_row_out, int64_t n,
+                          int m, int slot, double* partials, int max_partials, double* raw_gram, unsigned int* ticket,
+                          cudaStream_t st, int* launches) {
+    cudaError_t e =
+        dtype == QN_F32
+            ? qn::launch_row_t(static_cast<const float*>(window_g), static_cast<const float*>(g_col),
+                               static_cast<float*>(window_row_out), n, m, slot, partials, max_partials, raw_gram,
+                               ticket, st)
+            : qn::launch_row_t(static_cast<const __nv_bfloat16*>(window_g), static_cast<const __nv_bfloat16*>(g_col),
+                               static_cast<__nv_bfloat16*>(window_row_out), n, m, slot, partials, max_partials,
+                               raw_gram, ticket, st);
+    if (e == cudaSuccess && launches) *launches += 1;
+    return e;
+}

@@ -1,0 +1,320 @@
+// Single-CTA kernel between the two streaming passes: deterministic sum of the Gram partials, exact
+// m x m centring, two-sided Jacobi eigen-decomposition of G^T G in fp64, sigma_k, the lambda cut-off j
+// and the coefficient vector of the final combination.
+//
+// Paper, Section 2: V_G and Sigma_G come from the eigenpairs of G^H G; j is fixed by
+// sigma_j >= lambda sigma_1 > sigma_{j+1}; Eq. (4) with z = gbar needs alpha_k = gbar^T u_k and
+// alpha_k sigma_k^-1 y_k.  With w = G^T gbar one has alpha_k = v_k^T w / sigma_k, and both sums of
+// Eq. (4) collapse onto one m-vector d = sum_{k<=j} v_k (v_k^T w) / sigma_k^2:
+//     sum alpha_k u_k = G d,   sum alpha_k sigma_k^-1 y_k = Theta d.
+//
+// Centring: the streaming pass shifts each column by a reference r_i that only approximates the
+// mean.  With x' = g - r, C' = sum x' x'^T, t = sum x' r and P = I - 11^T/m:
+//     G^T G = P C' P,      G^T gbar = P t + P C' 1 / m,
+// exactly, for any r (r = 0 gives the raw Gram of the asynchronous window).
+#include "qn_device.cuh"
+
+namespace qn {
+
+constexpr int kLd = QN_MAX_M + 1;  // leading dimension of the shared matrices (odd: no bank conflicts)
+constexpr int kMaxSweeps = 30;
+
+struct SolveSmem {
+    double A[QN_MAX_M * kLd];
+    double V[QN_MAX_M * kLd];  // also scratch for the partial sums before the Jacobi phase
+    double w[QN_MAX_M];
+    double rowsum[QN_MAX_M];
+    double mu[QN_MAX_M];
+    double sigma[QN_MAX_M];
+    double rot_c[QN_MAX_M / 2], rot_s[QN_MAX_M / 2], rot_t[QN_MAX_M / 2];
+    double modec[QN_MAX_M];
+    double d[QN_MAX_M];
+    double red[32];
+    int order[QN_MAX_M];
+    int flag_nonfinite;
+    int flag_rotated;
+    int j;
+};
+
+__device__ __forceinline__ double block_sum(double x, double* red) {
+    // fixed-order block reduction; every thread returns the total
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    x = warp_sum(x);
+    __syncthreads();
+    if (lane == 0) red[warp] = x;
+    __syncthreads();
+    double s = 0.0;
+    for (int i = 0; i < nw; ++i) s += red[i];
+    return s;
+}
+
+// (p, q), p < q, of pair k in round r of the round-robin ordering over M2 (even) indices
+__device__ __forceinline__ void rr_pair(int M2, int r, int k, int& p, int& q) {
+    const int N = M2 - 1;
+    int a, b;
+    if (k == 0) {
+        a = N;
+        b = r;
+    } else {
+        a = (r + k) % N;
+        b = (r - k + N) % N;
+    }
+    p = a < b ? a : b;
+    q = a < b ? b : a;
+}
+
+__global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    SolveSmem& sm = *reinterpret_cast<SolveSmem*>(smem_raw);
+    const int m = prm.m;
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int tri_len = m * (m + 1) / 2;
+
+    if (tid == 0) {
+        sm.flag_nonfinite = 0;
+        sm.flag_rotated = 0;
+        sm.j = 0;
+    }
+    // ---------------------------------------------------------------- phase 1: C' and t
+    if (prm.source == QN_SRC_PARTIALS) {
+        const int E = tri_len + m;
+        double* packed = sm.V;  // E <= 2144 doubles fits in V (4160)
+        for (int e = tid; e < E; e += nthr) {
+            double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+            int p = 0;
+            for (; p + 3 < prm.num_partials; p += 4) {
+                s0 += prm.partials[(int64_t)(p + 0) * E + e];
+                s1 += prm.partials[(int64_t)(p + 1) * E + e];
+                s2 += prm.partials[(int64_t)(p + 2) * E + e];
+                s3 += prm.partials[(int64_t)(p + 3) * E + e];
+            }
+            for (; p < prm.num_partials; ++p) s0 += prm.partials[(int64_t)p * E + e];
+            packed[e] = (s0 + s1) + (s2 + s3);
+        }
+        __syncthreads();
+        for (int e = tid; e < m * m; e += nthr) {
+            const int k = e / m, l = e % m;
+            sm.A[k * kLd + l] = packed[k <= l ? qn_tri_index(m, k, l) : qn_tri_index(m, l, k)];
+        }
+        if (tid < m) sm.w[tid] = packed[tri_len + tid];
+        __syncthreads();
+        if (prm.raw_gram)
+            for (int e = tid; e < m * m; e += nthr) prm.raw_gram[e] = sm.A[(e / m) * kLd + (e % m)];
+    } else {
+        for (int e = tid; e < m * m; e += nthr) sm.A[(e / m) * kLd + (e % m)] = prm.raw_gram[e];
+        if (tid < m) sm.w[tid] = 0.0;
+        __syncthreads();
+    }
+
+    // ---------------------------------------------------------------- phase 2: exact centring
+    if (tid < m) {
+        double s = 0.0;
+        for (int l = 0; l < m; ++l) s += sm.A[tid * kLd + l];
+        sm.rowsum[tid] = s;
+    }
+    __syncthreads();
+    double tot = 0.0, tsum = 0.0;
+    for (int k = 0; k < m; ++k) {
+        tot += sm.rowsum[k];
+        tsum += sm.w[k];
+    }
+    const double inv_m = 1.0 / (double)m;
+    __syncthreads();
+    bool bad = false;
+    for (int e = tid; e < m * m; e += nthr) {
+        const int k = e / m, l = e % m;
+        const double c = sm.A[k * kLd + l] - (sm.rowsum[k] + sm.rowsum[l]) * inv_m + tot * inv_m * inv_m;
+        sm.A[k * kLd + l] = c;
+        bad |= !isfinite(c);
+        if (prm.gram_out) prm.gram_out[e] = c;
+    }
+    if (tid < m) {
+        const double wk = sm.w[tid] - tsum * inv_m + sm.rowsum[tid] * inv_m - tot * inv_m * inv_m;
+        bad |= !isfinite(wk);
+        // every thread has read w (tsum) before the barrier above; only thread tid rewrites w[tid]
+        sm.w[tid] = wk;
+        if (prm.gram_out) prm.gram_out[m * m + tid] = wk;
+    }
+    if (bad) sm.flag_nonfinite = 1;
+    __syncthreads();
+    if (prm.gram_only) {
+        if (tid == 0 && prm.result) {
+            prm.result->status = sm.flag_nonfinite ? QN_ERR_NONFINITE : QN_OK;
+            prm.result->j = 0;
+            prm.result->sweeps = 0;
+        }
+        return;
+    }
+    if (sm.flag_nonfinite) {  // the SGD update: no mode kept
+        if (tid < QN_MAX_M) {
+            prm.coef->c[tid] = 0.f;
+            prm.result->sigma[tid] = 0.0;
+        }
+        if (tid == 0) {
+            prm.coef->tau = (float)prm.tau;
+            prm.coef->inv_m = (float)inv_m;
+            prm.coef->m = m;
+            prm.result->j = 0;
+            prm.result->status = QN_ERR_NONFINITE;
+            prm.result->sweeps = 0;
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------------- phase 3: two-sided Jacobi
+    const int M2 = m + (m & 1);
+    const int H = M2 / 2;
+    if (M2 > m) {
+        for (int e = tid; e < M2; e += nthr) {
+            sm.A[m * kLd + e] = 0.0;
+            sm.A[e * kLd + m] = 0.0;
+        }
+    }
+    for (int e = tid; e < M2 * M2; e += nthr) sm.V[(e / M2) * kLd + (e % M2)] = (e / M2 == e % M2) ? 1.0 : 0.0;
+    __syncthreads();
+    double fro = 0.0;
+    for (int e = tid; e < m * m; e += nthr) {
+        const double a = sm.A[(e / m) * kLd + (e % m)];
+        fro += a * a;
+    }
+    fro = sqrt(block_sum(fro, sm.red));
+    const double thresh = 1e-15 * fro;
+    const int pa_idx = tid / H, pb_idx = tid % H;
+    const bool worker = tid < H * H;
+    int sweeps = 0;
+    bool converged = (fro == 0.0) || m < 2;
+    while (!converged && sweeps < kMaxSweeps) {
+        for (int r = 0; r < M2 - 1; ++r) {
+            int pa = 0, qa = 0, pb = 0, qb = 0;
+            if (worker) {
+                rr_pair(M2, r, pa_idx, pa, qa);
+                rr_pair(M2, r, pb_idx, pb, qb);
+                if (pa_idx == pb_idx) {
+                    const double apq = sm.A[pa * kLd + qa];
+                    double c = 1.0, s = 0.0, t = 0.0;
+                    if (fabs(apq) > thresh) {
+                        const double app = sm.A[pa * kLd + pa], aqq = sm.A[qa * kLd + qa];
+                        const double zeta = (aqq - app) / (2.0 * apq);
+                        t = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
+                        c = 1.0 / sqrt(1.0 + t * t);
+                        s = t * c;
+                        sm.flag_rotated = 1;
+                    }
+                    sm.rot_c[pa_idx] = c;
+                    sm.rot_s[pa_idx] = s;
+                    sm.rot_t[pa_idx] = t;
+                }
+            }
+            __syncthreads();
+            if (worker) {
+                const double ca = sm.rot_c[pa_idx], sa = sm.rot_s[pa_idx];
+                const double cb = sm.rot_c[pb_idx], sb = sm.rot_s[pb_idx];
+                const double x00 = sm.A[pa * kLd + pb], x01 = sm.A[pa * kLd + qb];
+                const double x10 = sm.A[qa * kLd + pb], x11 = sm.A[qa * kLd + qb];
+                double y00, y01, y10, y11;
+                if (pa_idx == pb_idx) {
+                    const double t = sm.rot_t[pa_idx];
+                    y00 = x00 - t * x01;
+                    y11 = x11 + t * x01;
+                    y01 = y10 = (sa == 0.0 && ca == 1.0) ? x01 : 0.0;  // untouched if the rotation was skipped
+                } else {
+                    const double t00 = cb * x00 - sb * x01, t01 = sb * x00 + cb * x01;
+                    const double t10 = cb * x10 - sb * x11, t11 = sb * x10 + cb * x11;
+                    y00 = ca * t00 - sa * t10;
+                    y10 = sa * t00 + ca * t10;
+                    y01 = ca * t01 - sa * t11;
+                    y11 = sa * t01 + ca * t11;
+                }
+                sm.A[pa * kLd + pb] = y00;
+                sm.A[pa * kLd + qb] = y01;
+                sm.A[qa * kLd + pb] = y10;
+                sm.A[qa * kLd + qb] = y11;
+                // V <- V J_b on rows 2*pa_idx, 2*pa_idx + 1
+#pragma unroll
+                for (int rr = 0; rr < 2; ++rr) {
+                    const int row = 2 * pa_idx + rr;
+                    const double v0 = sm.V[row * kLd + pb], v1 = sm.V[row * kLd + qb];
+                    sm.V[row * kLd + pb] = cb * v0 - sb * v1;
+                    sm.V[row * kLd + qb] = sb * v0 + cb * v1;
+                }
+            }
+            __syncthreads();
+        }
+        ++sweeps;
+        const int rotated = sm.flag_rotated;
+        __syncthreads();  // everyone has read the flag
+        if (!rotated) converged = true;
+        if (tid == 0) sm.flag_rotated = 0;
+        __syncthreads();  // reset is visible before the next sweep can set it again
+    }
+
+    // ---------------------------------------------------------------- phase 4: sigma, j, d, c
+    if (tid < m) sm.mu[tid] = sm.A[tid * kLd + tid];
+    __syncthreads();
+    if (tid < m) {
+        const double mine = sm.mu[tid];
+        int rank = 0;
+        for (int l = 0; l < m; ++l) {
+            const double o = sm.mu[l];
+            rank += (o > mine) || (o == mine && l < tid);
+        }
+        sm.order[rank] = tid;
+        sm.sigma[rank] = sqrt(mine > 0.0 ? mine : 0.0);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int j = 0;
+        const double s1 = sm.sigma[0];
+        if (s1 > 0.0)
+            for (int k = 0; k < m; ++k) j += (sm.sigma[k] >= prm.lambda * s1 && sm.sigma[k] > 0.0);
+        if (j > m - 1) j = m - 1;
+        sm.j = j;
+    }
+    __syncthreads();
+    const int j = sm.j;
+    if (tid < j) {
+        const int col = sm.order[tid];
+        double dot = 0.0;
+        for (int k = 0; k < m; ++k) dot += sm.V[k * kLd + col] * sm.w[k];
+        sm.modec[tid] = dot / sm.mu[col];
+    }
+    __syncthreads();
+    if (tid < m) {
+        double dk = 0.0;
+        for (int r = 0; r < j; ++r) dk += sm.V[tid * kLd + sm.order[r]] * sm.modec[r];
+        sm.d[tid] = dk;
+    }
+    __syncthreads();
+    if (tid < QN_MAX_M) {
+        double s = 0.0;
+        for (int k = 0; k < m; ++k) s += sm.d[k];
+        prm.coef->c[tid] = tid < m ? (float)(prm.tau * (sm.d[tid] - s * inv_m)) : 0.f;
+        prm.result->sigma[tid] = tid < m ? sm.sigma[tid] : 0.0;
+    }
+    if (tid == 0) {
+        prm.coef->tau = (float)prm.tau;
+        prm.coef->inv_m = (float)inv_m;
+        prm.coef->m = m;
+        prm.result->j = j;
+        prm.result->status = converged ? QN_OK : QN_ERR_NOT_CONVERGED;
+        prm.result->sweeps = sweeps;
+    }
+}
+
+}  // namespace qn
+
+cudaError_t qn_solve_init() {
+    return cudaFuncSetAttribute(qn::solve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)sizeof(qn::SolveSmem));
+}
+
+cudaError_t qn_launch_solve(const qn_solve_params& p, cudaStream_t st, int* launches) {
+    const int M2 = p.m + (p.m & 1);
+    const int H = M2 / 2;
+    int threads = 256;
+    while (threads < H * H) threads <<= 1;
+    qn::solve_kernel<<<1, threads, sizeof(qn::SolveSmem), st>>>(p);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess && launches) *launches += 1;
+    return e;
+}

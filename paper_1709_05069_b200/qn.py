@@ -1,0 +1,227 @@
+"""ctypes binding of libqn.so: the same entry points as ``include/qn.h``, arguments marshalled only.
+
+Tensors are ``torch`` CUDA tensors used purely as device memory (``data_ptr()``); streams are
+``torch.cuda`` streams passed by handle.  No arithmetic of the method happens in Python.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+QN_F32 = 0
+QN_BF16 = 1
+QN_MAX_M = 64
+
+QN_OK, QN_ERR_INVALID, QN_ERR_ALLOC, QN_ERR_CUDA, QN_ERR_STATE, QN_ERR_NOT_CONVERGED, QN_ERR_NONFINITE = range(7)
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libqn.so")
+_lib: Optional[ctypes.CDLL] = None
+
+EXPORTS = (
+    "qn_strerror", "qn_create", "qn_destroy", "qn_update", "qn_gram", "qn_push", "qn_update_window", "qn_rebuild",
+    "qn_window_alloc", "qn_window_theta", "qn_window_g", "qn_window_mark_full", "qn_update_host", "qn_status_sync",
+    "qn_last_launches", "qn_total_launches", "qn_last_sweeps",
+)
+
+
+class QNError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (status %d)" % (where, qn_strerror(status), status))
+
+
+def lib() -> ctypes.CDLL:
+    """Load libqn.so (built by ``paper_1709_05069_b200.build``).  Raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise FileNotFoundError(
+                "%s not found: build it with `python -m paper_1709_05069_b200.build` (there is no CPU fallback)" % _LIB_PATH)
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, i32, i64, dbl = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_double
+        L.qn_strerror.argtypes, L.qn_strerror.restype = [i32], ctypes.c_char_p
+        L.qn_create.argtypes, L.qn_create.restype = [i64, i32, i32, ctypes.POINTER(vp)], i32
+        L.qn_destroy.argtypes, L.qn_destroy.restype = [vp], i32
+        L.qn_update.argtypes, L.qn_update.restype = [vp, vp, vp, dbl, dbl, vp, vp, vp, vp], i32
+        L.qn_gram.argtypes, L.qn_gram.restype = [vp, vp, vp, vp], i32
+        L.qn_push.argtypes, L.qn_push.restype = [vp, i32, vp, vp, vp], i32
+        L.qn_update_window.argtypes, L.qn_update_window.restype = [vp, dbl, dbl, vp, vp, vp, vp], i32
+        L.qn_rebuild.argtypes, L.qn_rebuild.restype = [vp, vp], i32
+        L.qn_window_alloc.argtypes, L.qn_window_alloc.restype = [vp], i32
+        L.qn_window_theta.argtypes, L.qn_window_theta.restype = [vp], vp
+        L.qn_window_g.argtypes, L.qn_window_g.restype = [vp], vp
+        L.qn_window_mark_full.argtypes, L.qn_window_mark_full.restype = [vp], i32
+        L.qn_update_host.argtypes, L.qn_update_host.restype = [vp, vp, vp, dbl, dbl, vp, vp, vp, vp], i32
+        L.qn_status_sync.argtypes, L.qn_status_sync.restype = [vp], i32
+        L.qn_last_launches.argtypes, L.qn_last_launches.restype = [vp], i32
+        L.qn_total_launches.argtypes, L.qn_total_launches.restype = [vp], i64
+        L.qn_last_sweeps.argtypes, L.qn_last_sweeps.restype = [vp], i32
+        _lib = L
+    return _lib
+
+
+def qn_strerror(status: int) -> str:
+    return lib().qn_strerror(int(status)).decode()
+
+
+def _check(status: int, where: str, allow=()) -> int:
+    if status != QN_OK and status not in allow:
+        raise QNError(status, where)
+    return status
+
+
+def dtype_code(dtype: torch.dtype) -> int:
+    if dtype == torch.float32:
+        return QN_F32
+    if dtype == torch.bfloat16:
+        return QN_BF16
+    raise TypeError("storage dtype must be torch.float32 or torch.bfloat16")
+
+
+class Handle:
+    """Owner of a ``qn_handle``.  ``n``, ``m``, ``dtype`` as passed to ``qn_create``."""
+
+    def __init__(self, ptr: int, n: int, m: int, dtype: torch.dtype):
+        self.ptr, self.n, self.m, self.dtype = ptr, n, m, dtype
+
+    def close(self):
+        if self.ptr:
+            lib().qn_destroy(self.ptr)
+            self.ptr = 0
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    @property
+    def last_launches(self) -> int:
+        return lib().qn_last_launches(self.ptr)
+
+    @property
+    def total_launches(self) -> int:
+        return lib().qn_total_launches(self.ptr)
+
+    @property
+    def last_sweeps(self) -> int:
+        return lib().qn_last_sweeps(self.ptr)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _dev_matrix(t: torch.Tensor, h: Handle, name: str) -> int:
+    if not t.is_cuda or t.dtype != h.dtype or tuple(t.shape) != (h.m, h.n) or not t.is_contiguous():
+        raise ValueError("%s must be a contiguous CUDA tensor [m][n] of the handle's dtype" % name)
+    return t.data_ptr()
+
+
+def _dev_vector(t: torch.Tensor, h: Handle, name: str) -> int:
+    if not t.is_cuda or t.dtype != h.dtype or tuple(t.shape) != (h.n,) or not t.is_contiguous():
+        raise ValueError("%s must be a contiguous CUDA tensor [n] of the handle's dtype" % name)
+    return t.data_ptr()
+
+
+def qn_create(n: int, m: int, dtype: torch.dtype) -> Handle:
+    """Handle on the current CUDA device (``torch.cuda.current_device()``)."""
+    out = ctypes.c_void_p(0)
+    if torch.cuda.is_available():
+        torch.cuda.set_device(torch.cuda.current_device())  # make torch's device the runtime's current one
+    _check(lib().qn_create(int(n), int(m), dtype_code(dtype), ctypes.byref(out)), "qn_create")
+    return Handle(out.value, int(n), int(m), dtype)
+
+
+def qn_destroy(h: Handle) -> None:
+    h.close()
+
+
+def _host_outputs(h: Handle, want: bool):
+    if not want:
+        return None, None, None, None
+    j = ctypes.c_int32(0)
+    sigma = (ctypes.c_double * h.m)()
+    return j, sigma, ctypes.byref(j), ctypes.cast(sigma, ctypes.c_void_p)
+
+
+def qn_update(h: Handle, theta: torch.Tensor, g: torch.Tensor, tau: float, lam: float, theta_new: torch.Tensor,
+              want_host: bool = True, stream=None, allow=(QN_ERR_NOT_CONVERGED, QN_ERR_NONFINITE)):
+    """One Server step on device tensors.  Returns (j, sigma list, status) or None when ``want_host`` is False
+    (then nothing waits for the device)."""
+    j, sigma, jp, sp = _host_outputs(h, want_host)
+    st = lib().qn_update(h.ptr, _dev_matrix(theta, h, "theta"), _dev_matrix(g, h, "g"), float(tau), float(lam),
+                         _dev_vector(theta_new, h, "theta_new"), jp, sp, _stream_ptr(stream))
+    _check(st, "qn_update", allow)
+    if want_host:
+        return j.value, list(sigma), st
+    return None
+
+
+def qn_gram(h: Handle, g: torch.Tensor, gram_out: torch.Tensor, stream=None) -> None:
+    """Centred Gram (m*m) followed by w = G^T gbar (m) into ``gram_out`` (CUDA float64, m*m + m)."""
+    if not gram_out.is_cuda or gram_out.dtype != torch.float64 or gram_out.numel() != h.m * h.m + h.m \
+            or not gram_out.is_contiguous():
+        raise ValueError("gram_out must be a contiguous CUDA float64 tensor with m*m + m elements")
+    _check(lib().qn_gram(h.ptr, _dev_matrix(g, h, "g"), gram_out.data_ptr(), _stream_ptr(stream)), "qn_gram")
+
+
+def qn_push(h: Handle, slot: int, theta_col: torch.Tensor, g_col: torch.Tensor, stream=None) -> None:
+    _check(lib().qn_push(h.ptr, int(slot), _dev_vector(theta_col, h, "theta_col"), _dev_vector(g_col, h, "g_col"),
+                         _stream_ptr(stream)), "qn_push")
+
+
+def qn_update_window(h: Handle, tau: float, lam: float, theta_new: torch.Tensor, want_host: bool = True, stream=None,
+                     allow=(QN_ERR_NOT_CONVERGED, QN_ERR_NONFINITE)):
+    j, sigma, jp, sp = _host_outputs(h, want_host)
+    st = lib().qn_update_window(h.ptr, float(tau), float(lam), _dev_vector(theta_new, h, "theta_new"), jp, sp,
+                                _stream_ptr(stream))
+    _check(st, "qn_update_window", allow)
+    if want_host:
+        return j.value, list(sigma), st
+    return None
+
+
+def qn_rebuild(h: Handle, stream=None) -> None:
+    _check(lib().qn_rebuild(h.ptr, _stream_ptr(stream)), "qn_rebuild")
+
+
+def qn_window_alloc(h: Handle) -> None:
+    _check(lib().qn_window_alloc(h.ptr), "qn_window_alloc")
+
+
+def qn_window_ptrs(h: Handle) -> Tuple[int, int]:
+    return lib().qn_window_theta(h.ptr) or 0, lib().qn_window_g(h.ptr) or 0
+
+
+def qn_window_mark_full(h: Handle) -> None:
+    _check(lib().qn_window_mark_full(h.ptr), "qn_window_mark_full")
+
+
+def qn_update_host(h: Handle, theta_host: torch.Tensor, g_host: torch.Tensor, tau: float, lam: float,
+                   theta_new_host: torch.Tensor, stream=None, allow=(QN_ERR_NOT_CONVERGED, QN_ERR_NONFINITE)):
+    """The step with HOST tensors (pinned recommended): copies in, computes, copies theta_new out, waits."""
+    for t, shape, name in ((theta_host, (h.m, h.n), "theta_host"), (g_host, (h.m, h.n), "g_host"),
+                           (theta_new_host, (h.n,), "theta_new_host")):
+        if t.is_cuda or t.dtype != h.dtype or tuple(t.shape) != shape or not t.is_contiguous():
+            raise ValueError("%s must be a contiguous host tensor of shape %s and the handle's dtype" % (name, shape))
+    j, sigma, jp, sp = _host_outputs(h, True)
+    st = lib().qn_update_host(h.ptr, theta_host.data_ptr(), g_host.data_ptr(), float(tau), float(lam),
+                              theta_new_host.data_ptr(), jp, sp, _stream_ptr(stream))
+    _check(st, "qn_update_host", allow)
+    return j.value, list(sigma), st
+
+
+def qn_status_sync(h: Handle) -> int:
+    return lib().qn_status_sync(h.ptr)
