@@ -153,6 +153,25 @@ QN_API int64_t qn_total_launches(qn_handle h);
  * sigma_out non-NULL, or qn_status_sync), else -1. */
 QN_API int32_t qn_last_sweeps(qn_handle h);
 
+/*
+ * Per-kernel timing, for benchmarks.  Between qn_timing_begin and qn_timing_end every kernel the
+ * handle launches (up to max_kernels of them) is bracketed by two CUDA events recorded on the
+ * stream of the call.  qn_timing_end waits for those events and returns, per kind of kernel,
+ * the summed device time in milliseconds and the number of launches:
+ *   QN_TIME_GRAM     streaming Gram pass (means, centred Gram, G^T gbar; Section 2)
+ *   QN_TIME_SOLVE    single-CTA partial sum, centring, Jacobi, cut-off, coefficients
+ *   QN_TIME_COMBINE  streaming pass that writes theta_new (Eq. (2) with Eq. (4))
+ *   QN_TIME_ROW      one-row Gram refresh of the asynchronous window
+ * Timing is off by default and has no counterpart in the paper.
+ */
+#define QN_TIME_GRAM 0
+#define QN_TIME_SOLVE 1
+#define QN_TIME_COMBINE 2
+#define QN_TIME_ROW 3
+#define QN_TIME_KINDS 4
+QN_API qn_status qn_timing_begin(qn_handle h, int32_t max_kernels);
+QN_API qn_status qn_timing_end(qn_handle h, double ms_total[QN_TIME_KINDS], int32_t count[QN_TIME_KINDS]);
+
 #ifdef __cplusplus
 }
 #endif

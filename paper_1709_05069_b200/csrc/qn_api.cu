@@ -33,6 +33,11 @@ struct qn_ctx {
     void* stage_g;
     void* stage_out;
 
+    // optional per-kernel timing with CUDA events on the launching stream
+    cudaEvent_t* ev;       // 2 events per timed kernel
+    int32_t* ev_kind;
+    int32_t ev_cap, ev_used;
+
     cudaStream_t last_stream;
     int32_t last_launches;
     int64_t total_launches;
@@ -81,6 +86,23 @@ struct DeviceGuard {
 
 inline bool finite_d(double x) { return isfinite(x); }
 
+// Brackets one kernel launch with two events when timing is on (see qn_timing_begin).
+struct KernelTimer {
+    qn_handle h;
+    cudaStream_t st;
+    int idx = -1;
+    KernelTimer(qn_handle h_, cudaStream_t st_, int kind) : h(h_), st(st_) {
+        if (h->ev && h->ev_used < h->ev_cap) {
+            idx = h->ev_used++;
+            h->ev_kind[idx] = kind;
+            cudaEventRecord(h->ev[2 * idx], st);
+        }
+    }
+    ~KernelTimer() {
+        if (idx >= 0) cudaEventRecord(h->ev[2 * idx + 1], st);
+    }
+};
+
 inline void begin_call(qn_handle h, cudaStream_t st) {
     h->last_launches = 0;
     h->last_stream = st;
@@ -114,9 +136,12 @@ bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
 qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, double lambda, void* theta_new,
                    cudaStream_t st) {
     int np = 0;
-    if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st, &h->last_launches) !=
-        cudaSuccess)
-        return QN_ERR_CUDA;
+    {
+        KernelTimer t(h, st, QN_TIME_GRAM);
+        if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st,
+                           &h->last_launches) != cudaSuccess)
+            return QN_ERR_CUDA;
+    }
     qn_solve_params p;
     memset(&p, 0, sizeof(p));
     p.m = h->m;
@@ -127,9 +152,16 @@ qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, do
     p.lambda = lambda;
     p.coef = h->coef;
     p.result = h->result;
-    if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) return QN_ERR_CUDA;
-    if (qn_launch_combine(h->dtype, theta, g, h->n, h->m, h->coef, theta_new, st, &h->last_launches) != cudaSuccess)
-        return QN_ERR_CUDA;
+    {
+        KernelTimer t(h, st, QN_TIME_SOLVE);
+        if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) return QN_ERR_CUDA;
+    }
+    {
+        KernelTimer t(h, st, QN_TIME_COMBINE);
+        if (qn_launch_combine(h->dtype, theta, g, h->n, h->m, h->coef, theta_new, st, &h->last_launches) !=
+            cudaSuccess)
+            return QN_ERR_CUDA;
+    }
     return QN_OK;
 }
 
@@ -209,6 +241,11 @@ extern "C" qn_status qn_destroy(qn_handle h) {
     cudaFree(h->stage_g);
     cudaFree(h->stage_out);
     if (h->host_result) cudaFreeHost(h->host_result);
+    if (h->ev) {
+        for (int i = 0; i < 2 * h->ev_cap; ++i) cudaEventDestroy(h->ev[i]);
+        free(h->ev);
+        free(h->ev_kind);
+    }
     cudaGetLastError();
     delete h;
     return QN_OK;
@@ -297,9 +334,12 @@ extern "C" qn_status qn_push(qn_handle h, int32_t slot, const void* theta_col, c
     char* trow = static_cast<char*>(h->win_theta) + (size_t)slot * col_bytes;
     char* grow = static_cast<char*>(h->win_g) + (size_t)slot * col_bytes;
     if (cudaMemcpyAsync(trow, theta_col, col_bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess) s = QN_ERR_CUDA;
-    if (s == QN_OK && qn_launch_row(h->dtype, h->win_g, g_col, grow, h->n, h->m, slot, h->partials, h->max_partials,
-                                    h->raw_gram, h->ticket, st, &h->last_launches) != cudaSuccess)
-        s = QN_ERR_CUDA;
+    if (s == QN_OK) {
+        KernelTimer t(h, st, QN_TIME_ROW);
+        if (qn_launch_row(h->dtype, h->win_g, g_col, grow, h->n, h->m, slot, h->partials, h->max_partials,
+                          h->raw_gram, h->ticket, st, &h->last_launches) != cudaSuccess)
+            s = QN_ERR_CUDA;
+    }
     if (s == QN_OK) h->filled |= (1ull << slot);
     end_call(h);
     return s;
@@ -327,10 +367,16 @@ extern "C" qn_status qn_update_window(qn_handle h, double tau, double lambda, vo
     p.lambda = lambda;
     p.coef = h->coef;
     p.result = h->result;
-    if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) s = QN_ERR_CUDA;
-    if (s == QN_OK && qn_launch_combine(h->dtype, h->win_theta, h->win_g, h->n, h->m, h->coef, theta_new, st,
-                                        &h->last_launches) != cudaSuccess)
-        s = QN_ERR_CUDA;
+    {
+        KernelTimer t(h, st, QN_TIME_SOLVE);
+        if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) s = QN_ERR_CUDA;
+    }
+    if (s == QN_OK) {
+        KernelTimer t(h, st, QN_TIME_COMBINE);
+        if (qn_launch_combine(h->dtype, h->win_theta, h->win_g, h->n, h->m, h->coef, theta_new, st,
+                              &h->last_launches) != cudaSuccess)
+            s = QN_ERR_CUDA;
+    }
     end_call(h);
     if (s != QN_OK) return s;
     if (j_out || sigma_out) return fetch_result(h, st, j_out, sigma_out);
@@ -413,3 +459,61 @@ extern "C" qn_status qn_status_sync(qn_handle h) {
 extern "C" int32_t qn_last_launches(qn_handle h) { return h ? h->last_launches : 0; }
 extern "C" int64_t qn_total_launches(qn_handle h) { return h ? h->total_launches : 0; }
 extern "C" int32_t qn_last_sweeps(qn_handle h) { return h ? h->last_sweeps : -1; }
+
+extern "C" qn_status qn_timing_begin(qn_handle h, int32_t max_kernels) {
+    if (!h || max_kernels < 1 || max_kernels > (1 << 20)) return QN_ERR_INVALID;
+    if (h->ev) return QN_ERR_STATE;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return QN_ERR_CUDA;
+    cudaEvent_t* ev = static_cast<cudaEvent_t*>(calloc((size_t)2 * max_kernels, sizeof(cudaEvent_t)));
+    int32_t* kind = static_cast<int32_t*>(calloc((size_t)max_kernels, sizeof(int32_t)));
+    if (!ev || !kind) {
+        free(ev);
+        free(kind);
+        return QN_ERR_ALLOC;
+    }
+    for (int i = 0; i < 2 * max_kernels; ++i) {
+        if (cudaEventCreate(&ev[i]) != cudaSuccess) {
+            for (int k = 0; k < i; ++k) cudaEventDestroy(ev[k]);
+            free(ev);
+            free(kind);
+            cudaGetLastError();
+            return QN_ERR_CUDA;
+        }
+    }
+    h->ev_kind = kind;
+    h->ev_cap = max_kernels;
+    h->ev_used = 0;
+    h->ev = ev;
+    return QN_OK;
+}
+
+extern "C" qn_status qn_timing_end(qn_handle h, double ms_total[QN_TIME_KINDS], int32_t count[QN_TIME_KINDS]) {
+    if (!h || !ms_total || !count) return QN_ERR_INVALID;
+    if (!h->ev) return QN_ERR_STATE;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return QN_ERR_CUDA;
+    qn_status s = QN_OK;
+    for (int k = 0; k < QN_TIME_KINDS; ++k) {
+        ms_total[k] = 0.0;
+        count[k] = 0;
+    }
+    for (int i = 0; i < h->ev_used && s == QN_OK; ++i) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(h->ev[2 * i + 1]) != cudaSuccess ||
+            cudaEventElapsedTime(&ms, h->ev[2 * i], h->ev[2 * i + 1]) != cudaSuccess) {
+            s = QN_ERR_CUDA;
+            break;
+        }
+        ms_total[h->ev_kind[i]] += ms;
+        count[h->ev_kind[i]] += 1;
+    }
+    for (int i = 0; i < 2 * h->ev_cap; ++i) cudaEventDestroy(h->ev[i]);
+    free(h->ev);
+    free(h->ev_kind);
+    h->ev = nullptr;
+    h->ev_kind = nullptr;
+    h->ev_cap = h->ev_used = 0;
+    cudaGetLastError();
+    return s;
+}

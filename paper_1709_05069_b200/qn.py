@@ -23,8 +23,9 @@ _lib: Optional[ctypes.CDLL] = None
 EXPORTS = (
     "qn_strerror", "qn_create", "qn_destroy", "qn_update", "qn_gram", "qn_push", "qn_update_window", "qn_rebuild",
     "qn_window_alloc", "qn_window_theta", "qn_window_g", "qn_window_mark_full", "qn_update_host", "qn_status_sync",
-    "qn_last_launches", "qn_total_launches", "qn_last_sweeps",
+    "qn_last_launches", "qn_total_launches", "qn_last_sweeps", "qn_timing_begin", "qn_timing_end",
 )
+TIME_KINDS = ("gram", "solve", "combine", "row")
 
 
 class QNError(RuntimeError):
@@ -59,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.qn_last_launches.argtypes, L.qn_last_launches.restype = [vp], i32
         L.qn_total_launches.argtypes, L.qn_total_launches.restype = [vp], i64
         L.qn_last_sweeps.argtypes, L.qn_last_sweeps.restype = [vp], i32
+        L.qn_timing_begin.argtypes, L.qn_timing_begin.restype = [vp, i32], i32
+        L.qn_timing_end.argtypes, L.qn_timing_end.restype = [vp, vp, vp], i32
         _lib = L
     return _lib
 
@@ -225,3 +228,16 @@ def qn_update_host(h: Handle, theta_host: torch.Tensor, g_host: torch.Tensor, ta
 
 def qn_status_sync(h: Handle) -> int:
     return lib().qn_status_sync(h.ptr)
+
+
+def qn_timing_begin(h: Handle, max_kernels: int) -> None:
+    _check(lib().qn_timing_begin(h.ptr, int(max_kernels)), "qn_timing_begin")
+
+
+def qn_timing_end(h: Handle):
+    """{kind: (total_ms, launches)} for the kernels launched since ``qn_timing_begin``."""
+    ms = (ctypes.c_double * len(TIME_KINDS))()
+    cnt = (ctypes.c_int32 * len(TIME_KINDS))()
+    _check(lib().qn_timing_end(h.ptr, ctypes.cast(ms, ctypes.c_void_p), ctypes.cast(cnt, ctypes.c_void_p)),
+           "qn_timing_end")
+    return {k: (ms[i], cnt[i]) for i, k in enumerate(TIME_KINDS)}

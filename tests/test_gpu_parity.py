@@ -52,7 +52,13 @@ def check_against_oracle(qn, theta, g, tau, lam, dtype, expect_j=None, sample=No
     if sample is not None:
         got = got[sample]
     rel = np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new)
-    assert rel <= TOL[dtype], rel
+    if dtype == "bf16" and len(got) < 64:
+        # With a handful of elements the L2 figure is not an average: one bf16 rounding is off by up to
+        # 2^-9 relative, and an fp32-vs-fp64 difference next to a rounding boundary can move the result to
+        # the neighbouring bf16 value.  Bound every element by one bf16 ulp (2^-8 relative, 2^-133 absolute).
+        assert np.all(np.abs(got - ref.theta_new) <= 2.0 ** -8 * np.abs(ref.theta_new) + 2.0 ** -133)
+    else:
+        assert rel <= TOL[dtype], rel
     return rel, j, out
 
 
