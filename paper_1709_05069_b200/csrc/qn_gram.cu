@@ -4,14 +4,23 @@
 // and the numerators of alpha_k for z = gbar.)  The solve kernel sums the partials in a fixed
 // order and applies the exact m x m centring, so any rounding in the per-column reference cancels.
 //
-// Arithmetic: fp32 products, fp32 accumulation over at most kFlushCols columns per thread, then
-// fp64.  Every thread owns fixed columns and fixed output entries, so results are bitwise
-// reproducible for a given grid.
+// Arithmetic, three modes:
+//   kFast     fp32 products, fp32 accumulation over at most kFlushCols columns per thread, then fp64.
+//             The rounding errors of the products are unbiased and average out as 1/sqrt(n); used
+//             for n >= QN_PRECISE_BELOW, where they stay below 1e-10 of the largest eigenvalue.
+//   kPrecise  the shifted values are rounded to fp32 once, every product and sum is fp64 (a product of
+//             two fp32 values is exact in fp64), so the result is the exact Gram of slightly perturbed
+//             data and stays positive semi-definite to fp64 accuracy; used for small n.
+//   kRaw      as kPrecise with reference 0: the raw Gram of the asynchronous window, which has to
+//             carry the cancellation of the later m x m centring.
+// Every thread owns fixed columns and fixed output entries, so results are bitwise reproducible for
+// a given grid.
 #include "qn_device.cuh"
 
 namespace qn {
 
 constexpr int kThreads = 256;
+enum GramMode { kFast = 0, kPrecise = 1, kRaw = 2 };
 constexpr int kFlushCols = 32;  // columns accumulated in fp32 by one thread between fp64 flushes
 
 // ------------------------------------------------------------------------------------------------
@@ -46,7 +55,7 @@ struct DirectItem {
     }
 };
 
-template <typename T, bool kAligned, bool kRaw>
+template <typename T, bool kAligned, int kMode>
 __global__ void __launch_bounds__(kThreads, 1)
 gram_direct_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ partials) {
     using Item = DirectItem<T, kAligned>;
@@ -84,19 +93,24 @@ gram_direct_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict
                 x[k] = cur.get(k, e);
                 s += x[k];
             }
-            if (kRaw) {
-                // raw Gram (reference 0), accumulated directly in fp64: products of fp32 or bf16
-                // values are exact in fp64
+            const float r = kMode == kRaw ? 0.f : s * inv_m;
+#pragma unroll
+            for (int k = 0; k < kDirectM; ++k) x[k] = fmaf(-mask[k], r, x[k]);
+            if (kMode != kFast) {
+                double xd[kDirectM];
+#pragma unroll
+                for (int k = 0; k < kDirectM; ++k) xd[k] = (double)x[k];
 #pragma unroll
                 for (int k = 0, idx = 0; k < kDirectM; ++k) {
-                    const double xk = (double)x[k];
 #pragma unroll
-                    for (int l = k; l < kDirectM; ++l, ++idx) acc64[idx] = fma(xk, (double)x[l], acc64[idx]);
+                    for (int l = k; l < kDirectM; ++l, ++idx) acc64[idx] = fma(xd[k], xd[l], acc64[idx]);
+                }
+                if (kMode == kPrecise) {
+                    const double rd = (double)r;
+#pragma unroll
+                    for (int k = 0; k < kDirectM; ++k) acc64[kDirectTri + k] = fma(xd[k], rd, acc64[kDirectTri + k]);
                 }
             } else {
-                const float r = s * inv_m;
-#pragma unroll
-                for (int k = 0; k < kDirectM; ++k) x[k] = fmaf(-mask[k], r, x[k]);
 #pragma unroll
                 for (int k = 0, idx = 0; k < kDirectM; ++k) {
 #pragma unroll
@@ -106,7 +120,7 @@ gram_direct_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict
                 for (int k = 0; k < kDirectM; ++k) acc[kDirectTri + k] = fmaf(x[k], r, acc[kDirectTri + k]);
             }
         }
-        if (!kRaw && ++iters == kFlushIters) {
+        if (kMode == kFast && ++iters == kFlushIters) {
             iters = 0;
 #pragma unroll
             for (int e = 0; e < kDirectAcc; ++e) {
@@ -116,7 +130,7 @@ gram_direct_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict
         }
         cur = nxt;
     }
-    if (!kRaw) {
+    if (kMode == kFast) {
 #pragma unroll
         for (int e = 0; e < kDirectAcc; ++e) acc64[e] += (double)acc[e];
     }
@@ -168,7 +182,7 @@ struct TiledSmem {
     float psum[kTileCols * 17];
 };
 
-template <typename T, bool kAligned, bool kRaw>
+template <typename T, bool kAligned, int kMode>
 __global__ void __launch_bounds__(kThreads, 1)
 gram_tiled_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ partials) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -245,9 +259,9 @@ gram_tiled_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict_
         for (int e = 0; e < kCols; ++e) {
             float s = 0.f;
             for (int q = 0; q < kRowGroups; ++q) s += sm.psum[(cg * kCols + e) * (kRowGroups + 1) + q];
-            r[e] = kRaw ? 0.f : s * inv_m;
+            r[e] = kMode == kRaw ? 0.f : s * inv_m;
         }
-        if (!kRaw) {
+        if (kMode != kRaw) {
             for (int k = rg; k < m; k += kRowGroups) {
 #pragma unroll
                 for (int e = 0; e < kCols; ++e) sm.xs[(cg * kCols + e) * RBP + k] -= r[e];
@@ -269,25 +283,42 @@ gram_tiled_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict_
                 const float4 b0 = rec[2 * tb], b1 = rec[2 * tb + 1];
                 const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
                 const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                if (kMode == kFast) {
 #pragma unroll
-                for (int p = 0; p < 8; ++p)
+                    for (int p = 0; p < 8; ++p)
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) acc[p * 8 + q] = fmaf(a[p], b[q], acc[p * 8 + q]);
+                        for (int q = 0; q < 8; ++q) acc[p * 8 + q] = fmaf(a[p], b[q], acc[p * 8 + q]);
+                } else {
+                    double ad[8], bd[8];
+#pragma unroll
+                    for (int p = 0; p < 8; ++p) {
+                        ad[p] = (double)a[p];
+                        bd[p] = (double)b[p];
+                    }
+#pragma unroll
+                    for (int p = 0; p < 8; ++p)
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) acc64[p * 8 + q] = fma(ad[p], bd[q], acc64[p * 8 + q]);
+                }
             }
         }
-        cols_since_flush += kTileCols / colstep;
-        if (kRaw || cols_since_flush >= kFlushCols) {
-            cols_since_flush = 0;
+        if (kMode == kFast) {
+            cols_since_flush += kTileCols / colstep;
+            if (cols_since_flush >= kFlushCols) {
+                cols_since_flush = 0;
 #pragma unroll
-            for (int e = 0; e < 64; ++e) {
-                acc64[e] += (double)acc[e];
-                acc[e] = 0.f;
+                for (int e = 0; e < 64; ++e) {
+                    acc64[e] += (double)acc[e];
+                    acc[e] = 0.f;
+                }
             }
         }
         __syncthreads();
     }
+    if (kMode == kFast) {
 #pragma unroll
-    for (int e = 0; e < 64; ++e) acc64[e] += (double)acc[e];
+        for (int e = 0; e < 64; ++e) acc64[e] += (double)acc[e];
+    }
 
     // CTA reduction: for each block, sum the kThreads/S column classes in the order 0,1,2,...
     double* red = reinterpret_cast<double*>(smem_raw);  // reuse of the tile storage: kThreads*16 doubles
@@ -318,43 +349,44 @@ gram_tiled_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict_
 // ------------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------------
+template <typename T, bool kAligned, int kMode>
+static cudaError_t launch_gram_mode(const T* g, int64_t n, int m, double* partials, int grid, cudaStream_t st) {
+    if (m <= kDirectM) {
+        gram_direct_kernel<T, kAligned, kMode><<<grid, kThreads, 0, st>>>(g, n, m, partials);
+        return cudaGetLastError();
+    }
+    auto kern = gram_tiled_kernel<T, kAligned, kMode>;
+    const size_t smem = sizeof(TiledSmem);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, kThreads, smem, st>>>(g, n, m, partials);
+    return cudaGetLastError();
+}
+
 template <typename T>
 static cudaError_t launch_gram_t(const T* g, int64_t n, int m, bool raw, double* partials, int* num_partials,
                                  int max_partials, cudaStream_t st) {
     const bool aligned = (reinterpret_cast<uintptr_t>(g) % 16 == 0) && ((n * (int64_t)sizeof(T)) % 16 == 0);
     const int sms = qn_sm_count();
+    int64_t ntiles;
     if (m <= kDirectM) {
         const int64_t nitems = aligned ? n / Storage<T>::kVec : n;
-        const int64_t ntiles = (nitems + kThreads - 1) / kThreads;
-        int grid = (int)(ntiles < sms ? ntiles : sms);
-        if (grid > max_partials) grid = max_partials;
-        *num_partials = grid;
-        if (aligned) {
-            if (raw)
-                gram_direct_kernel<T, true, true><<<grid, kThreads, 0, st>>>(g, n, m, partials);
-            else
-                gram_direct_kernel<T, true, false><<<grid, kThreads, 0, st>>>(g, n, m, partials);
-        } else {
-            if (raw)
-                gram_direct_kernel<T, false, true><<<grid, kThreads, 0, st>>>(g, n, m, partials);
-            else
-                gram_direct_kernel<T, false, false><<<grid, kThreads, 0, st>>>(g, n, m, partials);
-        }
-        return cudaGetLastError();
+        ntiles = (nitems + kThreads - 1) / kThreads;
+    } else {
+        ntiles = (n + kTileCols - 1) / kTileCols;
     }
-    const int64_t ntiles = (n + kTileCols - 1) / kTileCols;
     int grid = (int)(ntiles < sms ? ntiles : sms);
     if (grid > max_partials) grid = max_partials;
     *num_partials = grid;
-    const size_t smem = sizeof(TiledSmem);
-    auto go = [&](auto kern) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        kern<<<grid, kThreads, smem, st>>>(g, n, m, partials);
-        return cudaGetLastError();
-    };
-    if (aligned) return raw ? go(gram_tiled_kernel<T, true, true>) : go(gram_tiled_kernel<T, true, false>);
-    return raw ? go(gram_tiled_kernel<T, false, true>) : go(gram_tiled_kernel<T, false, false>);
+    const int mode = raw ? kRaw : (n < QN_PRECISE_BELOW ? kPrecise : kFast);
+    if (aligned) {
+        if (mode == kRaw) return launch_gram_mode<T, true, kRaw>(g, n, m, partials, grid, st);
+        if (mode == kPrecise) return launch_gram_mode<T, true, kPrecise>(g, n, m, partials, grid, st);
+        return launch_gram_mode<T, true, kFast>(g, n, m, partials, grid, st);
+    }
+    if (mode == kRaw) return launch_gram_mode<T, false, kRaw>(g, n, m, partials, grid, st);
+    if (mode == kPrecise) return launch_gram_mode<T, false, kPrecise>(g, n, m, partials, grid, st);
+    return launch_gram_mode<T, false, kFast>(g, n, m, partials, grid, st);
 }
 
 }  // namespace qn

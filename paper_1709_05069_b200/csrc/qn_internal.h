@@ -13,6 +13,15 @@
 __host__ __device__ inline int qn_tri_index(int m, int k, int l) { return k * m - (k * (k - 1)) / 2 + (l - k); }
 __host__ __device__ inline int qn_partial_len(int m) { return m * (m + 1) / 2 + m; }
 
+// Below this n the Gram pass forms every product and sum in fp64 (see qn_gram.cu): with fp32 products
+// the error of an eigenvalue is about 6e-8 * mu_1 / sqrt(n), which only falls under the 1e-10 * mu_1
+// needed for sigma to be good to 1e-5 * sigma_1 on near-null modes once n is a few million.
+#define QN_PRECISE_BELOW (int64_t(1) << 22)
+
+// Eigenvalues of the centred Gram below this fraction of the largest diagonal entry of the
+// uncentred (reference-shifted or raw) Gram are rounding noise of the m x m centring and are set to 0.
+#define QN_NOISE_FLOOR 1.4e-14
+
 // Device block read back by the host after a step.
 struct qn_result_block {
     int32_t j;

@@ -30,6 +30,7 @@ struct SolveSmem {
     double modec[QN_MAX_M];
     double d[QN_MAX_M];
     double red[32];
+    double diag_scale;  // largest diagonal entry of the uncentred Gram
     int order[QN_MAX_M];
     int flag_nonfinite;
     int flag_rotated;
@@ -113,11 +114,13 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
         sm.rowsum[tid] = s;
     }
     __syncthreads();
-    double tot = 0.0, tsum = 0.0;
+    double tot = 0.0, tsum = 0.0, dmax = 0.0;
     for (int k = 0; k < m; ++k) {
         tot += sm.rowsum[k];
         tsum += sm.w[k];
+        dmax = fmax(dmax, sm.A[k * kLd + k]);
     }
+    if (tid == 0) sm.diag_scale = dmax;
     const double inv_m = 1.0 / (double)m;
     __syncthreads();
     bool bad = false;
@@ -249,7 +252,10 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
     }
 
     // ---------------------------------------------------------------- phase 4: sigma, j, d, c
-    if (tid < m) sm.mu[tid] = sm.A[tid * kLd + tid];
+    if (tid < m) {
+        const double mu = sm.A[tid * kLd + tid];
+        sm.mu[tid] = mu > QN_NOISE_FLOOR * sm.diag_scale ? mu : 0.0;
+    }
     __syncthreads();
     if (tid < m) {
         const double mine = sm.mu[tid];

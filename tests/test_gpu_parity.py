@@ -52,11 +52,22 @@ def check_against_oracle(qn, theta, g, tau, lam, dtype, expect_j=None, sample=No
     if sample is not None:
         got = got[sample]
     rel = np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new)
-    if dtype == "bf16" and len(got) < 64:
-        # With a handful of elements the L2 figure is not an average: one bf16 rounding is off by up to
-        # 2^-9 relative, and an fp32-vs-fp64 difference next to a rounding boundary can move the result to
-        # the neighbouring bf16 value.  Bound every element by one bf16 ulp (2^-8 relative, 2^-133 absolute).
-        assert np.all(np.abs(got - ref.theta_new) <= 2.0 ** -8 * np.abs(ref.theta_new) + 2.0 ** -133)
+    if len(got) < 64:
+        # With a handful of elements the L2 figure is not an average.  Bound every element instead: the
+        # fp32 combination is accurate to 1e-5 of the magnitude of the terms it adds (thetabar, tau*z_perp
+        # and tau*sum alpha_k y_k / sigma_k, which may cancel), and for bf16 storage the single output
+        # rounding adds at most one bf16 ulp (2^-8 relative, 2^-133 absolute).
+        t64, g64 = oracle.storage_to_f64(tb), oracle.storage_to_f64(gb)
+        U, Y, sg, jj = oracle.left_vectors(tb, gb, lam)
+        al = ref.alpha[:jj]
+        scale = np.abs(t64.mean(0)) + abs(tau) * (np.abs(g64.mean(0)) + np.abs(U) @ np.abs(al)
+                                                  + np.abs(Y) @ np.abs(al / sg[:jj]))
+        if sample is not None:
+            scale = scale[sample]
+        bound = 1e-5 * scale
+        if dtype == "bf16":
+            bound = bound + 2.0 ** -8 * np.abs(ref.theta_new) + 2.0 ** -133
+        assert np.all(np.abs(got - ref.theta_new) <= bound), (got, ref.theta_new, bound)
     else:
         assert rel <= TOL[dtype], rel
     return rel, j, out
@@ -267,7 +278,8 @@ def test_async_window_matches_sync_oracle(qn, dtype, m, n, writes):
         qn.qn_rebuild(h)
         j2, s2, _ = qn.qn_update_window(h, cfg.tau, cfg.lam, out)
         assert j1 == j2
-        np.testing.assert_allclose(s1, s2, rtol=1e-9, atol=1e-9 * s1[0])
+        # the last sigma is the square root of round-off (about 1e-8 sigma_1) and differs between the two routes
+        np.testing.assert_allclose(s1, s2, rtol=1e-9, atol=1e-6 * s1[0])
         assert torch.linalg.norm(a.double() - out.double()) <= 1e-6 * torch.linalg.norm(out.double())
 
 
