@@ -154,6 +154,36 @@ QN_API int64_t qn_total_launches(qn_handle h);
 QN_API int32_t qn_last_sweeps(qn_handle h);
 
 /*
+ * qn_gram without any allocation (the paper has no counterpart; this exists for deployment).
+ *
+ * For callers that may not allocate device memory once they are running -- code living inside a
+ * framework whose caching allocator owns all of the GPU's memory, services with a no-allocation
+ * rule after start-up because cudaMalloc can block, synchronise the device or fail late, plug-ins
+ * that are only ever handed buffers -- and therefore cannot use qn_create.  It needs no handle:
+ * the caller passes the input g ([m][n], DEVICE, as for qn_gram) and the output gram_out
+ * (DEVICE, m*m + m doubles: centred Gram, then G^T gbar), and the per-CTA partial sums that the
+ * pass keeps between its two kernels go to a fixed array of 716,800 bytes compiled into the
+ * library, which each GPU that loads the library holds until the process exits.
+ *
+ * Limits: 1 <= m <= QN_STATIC_MAX_M (32); a larger m does not fit the fixed array and is rejected
+ * with QN_ERR_INVALID before anything is launched.  n is unlimited.  Runs on the CURRENT device.
+ * The call makes no cudaMalloc/cudaFree and calls no allocating routine; it only enqueues two
+ * kernels on cuda_stream and returns.
+ *
+ * First call on each device: looks up the array's device address (and raises one kernel's
+ * shared-memory limit).  Make that first call during start-up, before any stream capture.
+ *
+ * Sharing: all calls on a device use the same array, and it keeps whatever the previous call left
+ * there.  Each call overwrites every entry it later reads, so nothing needs clearing and results
+ * do not depend on earlier calls; but two calls whose kernels can overlap on the GPU (different
+ * streams, no ordering between them) race on the array and give wrong results -- order them.
+ */
+#define QN_STATIC_MAX_M 32
+#define QN_STATIC_MAX_CTAS 160
+QN_API qn_status qn_gram_static(int64_t n, int32_t m, qn_dtype dtype, const void* g, double* gram_out,
+                                void* cuda_stream);
+
+/*
  * Per-kernel timing, for benchmarks.  Between qn_timing_begin and qn_timing_end every kernel the
  * handle launches (up to max_kernels of them) is bracketed by two CUDA events recorded on the
  * stream of the call.  qn_timing_end waits for those events and returns, per kind of kernel,

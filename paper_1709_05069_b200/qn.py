@@ -24,6 +24,7 @@ EXPORTS = (
     "qn_strerror", "qn_create", "qn_destroy", "qn_update", "qn_gram", "qn_push", "qn_update_window", "qn_rebuild",
     "qn_window_alloc", "qn_window_theta", "qn_window_g", "qn_window_mark_full", "qn_update_host", "qn_status_sync",
     "qn_last_launches", "qn_total_launches", "qn_last_sweeps", "qn_timing_begin", "qn_timing_end",
+    "qn_gram_static",
 )
 TIME_KINDS = ("gram", "solve", "combine", "row")
 
@@ -60,6 +61,7 @@ def lib() -> ctypes.CDLL:
         L.qn_last_launches.argtypes, L.qn_last_launches.restype = [vp], i32
         L.qn_total_launches.argtypes, L.qn_total_launches.restype = [vp], i64
         L.qn_last_sweeps.argtypes, L.qn_last_sweeps.restype = [vp], i32
+        L.qn_gram_static.argtypes, L.qn_gram_static.restype = [i64, i32, i32, vp, vp, vp], i32
         L.qn_timing_begin.argtypes, L.qn_timing_begin.restype = [vp, i32], i32
         L.qn_timing_end.argtypes, L.qn_timing_end.restype = [vp, vp, vp], i32
         _lib = L
@@ -241,3 +243,21 @@ def qn_timing_end(h: Handle):
     _check(lib().qn_timing_end(h.ptr, ctypes.cast(ms, ctypes.c_void_p), ctypes.cast(cnt, ctypes.c_void_p)),
            "qn_timing_end")
     return {k: (ms[i], cnt[i]) for i, k in enumerate(TIME_KINDS)}
+
+
+QN_STATIC_MAX_M = 32
+
+
+def qn_gram_static(g: torch.Tensor, gram_out: torch.Tensor, stream=None) -> None:
+    """``qn_gram`` for callers that must not allocate: no handle, scratch in a fixed array inside the library.
+
+    ``g`` is a contiguous CUDA tensor [m][n] (float32 or bfloat16, m <= 32), ``gram_out`` a CUDA float64
+    tensor with m*m + m elements.  Calls on one device share the scratch: do not let two overlap."""
+    if not g.is_cuda or g.dim() != 2 or not g.is_contiguous():
+        raise ValueError("g must be a contiguous CUDA tensor [m][n]")
+    m, n = g.shape
+    if not gram_out.is_cuda or gram_out.dtype != torch.float64 or gram_out.numel() != m * m + m \
+            or not gram_out.is_contiguous():
+        raise ValueError("gram_out must be a contiguous CUDA float64 tensor with m*m + m elements")
+    _check(lib().qn_gram_static(int(n), int(m), dtype_code(g.dtype), g.data_ptr(), gram_out.data_ptr(),
+                                _stream_ptr(stream)), "qn_gram_static")

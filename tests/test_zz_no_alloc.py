@@ -1,0 +1,65 @@
+"""The allocation-free Gram entry point, qn_gram_static, against the handle-based qn_gram.
+
+Collected last on purpose (file name): a run that stops at the first failure has then already run
+every other test.  The entry point serves callers that cannot allocate device memory while running
+(inside a framework whose allocator owns the GPU's memory, or under a no-cudaMalloc-after-start-up
+rule), so the test also checks that calling it leaves the CUDA context's allocated memory unchanged.
+"""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("dtype,m,n", [("f32", 8, 300_001), ("bf16", 16, 200_000), ("f32", 32, 5_000_000)])
+def test_static_gram_matches_handle_gram_twice(dtype, m, n):
+    from paper_1709_05069_b200 import qn
+
+    assert torch.cuda.is_available()
+    outs_static, outs_handle = [], []
+    # two calls in a row on different inputs: the second must not be affected by what the first left
+    # in the shared scratch array
+    for call in range(2):
+        cfg = W.Config(20 + call, n, m, dtype, -1, 1, 0, 0.05, 1e-3, 0.5, 0.05)
+        _, g = W.generate(cfg, "cuda")
+        a = torch.full((m * m + m,), float("nan"), dtype=torch.float64, device="cuda")
+        b = torch.full((m * m + m,), float("nan"), dtype=torch.float64, device="cuda")
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
+        qn.qn_gram_static(g, a)
+        torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        if call == 1:  # the first call on a device may load the module that holds the array
+            assert free_after == free_before
+        with qn.qn_create(n, m, g.dtype) as h:
+            qn.qn_gram(h, g, b)
+            torch.cuda.synchronize()
+        outs_static.append(a.cpu().numpy())
+        outs_handle.append(b.cpu().numpy())
+    for a, b in zip(outs_static, outs_handle):
+        assert np.all(np.isfinite(a))
+        scale = np.abs(b[: m * m]).max()
+        assert np.max(np.abs(a[: m * m] - b[: m * m])) <= 2e-9 * scale  # the Gram tolerance of test_gram_entry_point
+        wscale = max(np.abs(b[m * m:]).max(), 1e-300)
+        assert np.max(np.abs(a[m * m:] - b[m * m:])) <= 1e-7 * wscale
+    assert not np.array_equal(outs_static[0], outs_static[1])
+
+
+def test_static_gram_rejects_sizes_beyond_its_scratch():
+    from paper_1709_05069_b200 import qn
+
+    L = qn.lib()
+    g = torch.zeros(33, 64, device="cuda")
+    out = torch.zeros(33 * 33 + 33, dtype=torch.float64, device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+    assert L.qn_gram_static(64, 33, 0, g.data_ptr(), out.data_ptr(), st) == qn.QN_ERR_INVALID
+    assert L.qn_gram_static(0, 8, 0, g.data_ptr(), out.data_ptr(), st) == qn.QN_ERR_INVALID
+    assert L.qn_gram_static(64, 8, 0, None, out.data_ptr(), st) == qn.QN_ERR_INVALID
+    assert L.qn_gram_static(64, 8, 5, g.data_ptr(), out.data_ptr(), st) == qn.QN_ERR_INVALID
+    with pytest.raises(qn.QNError):
+        qn.qn_gram_static(g, out)
