@@ -66,7 +66,8 @@ typedef enum {
     QN_ERR_CUDA = 3,          /* a CUDA runtime call failed (no device, launch error, ...) */
     QN_ERR_STATE = 4,         /* call not valid in the handle's state (window not full, ...) */
     QN_ERR_NOT_CONVERGED = 5, /* Jacobi hit its sweep limit; results were still written */
-    QN_ERR_NONFINITE = 6      /* Gram contained NaN/Inf; theta_new written with j = 0 */
+    QN_ERR_NONFINITE = 6,     /* Gram contained NaN/Inf; theta_new written with j = 0 */
+    QN_ERR_DEVICE_TIMEOUT = 7 /* a kernel's bounded wait ran out; theta_new written with j = 0 */
 } qn_status;
 
 /* Human-readable text for a status code (static storage, never NULL). */

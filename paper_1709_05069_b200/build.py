@@ -10,7 +10,7 @@ _CSRC = os.path.join(_PKG, "csrc")
 _INCLUDE = os.path.join(os.path.dirname(_PKG), "include")
 LIB_PATH = os.path.join(_PKG, "libqn.so")
 
-SOURCES = ["qn_api.cu", "qn_gram.cu", "qn_solve.cu", "qn_combine.cu", "qn_row.cu", "qn_static.cu"]
+SOURCES = ["qn_api.cu", "qn_gram.cu", "qn_solve.cu", "qn_combine.cu", "qn_row.cu", "qn_static.cu", "qn_gram_tc.cu"]
 HEADERS = ["qn_internal.h", "qn_device.cuh"]
 
 NVCC_FLAGS = [

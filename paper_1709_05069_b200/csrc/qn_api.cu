@@ -20,6 +20,7 @@ struct qn_ctx {
     qn_result_block* result;      // device
     qn_result_block* host_result; // pinned host
     unsigned int* ticket;         // device, zero between launches
+    int* error_word;              // device, set by a kernel that gave up on a bounded wait
 
     // asynchronous window
     void* win_theta;
@@ -65,6 +66,7 @@ extern "C" const char* qn_strerror(qn_status s) {
         case QN_ERR_STATE: return "call not valid in this state";
         case QN_ERR_NOT_CONVERGED: return "Jacobi sweep limit reached";
         case QN_ERR_NONFINITE: return "non-finite Gram";
+        case QN_ERR_DEVICE_TIMEOUT: return "device wait limit reached";
     }
     return "unknown status";
 }
@@ -139,7 +141,7 @@ qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, do
     {
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st,
-                           &h->last_launches) != cudaSuccess)
+                           &h->last_launches, h->error_word) != cudaSuccess)
             return QN_ERR_CUDA;
     }
     qn_solve_params p;
@@ -152,6 +154,7 @@ qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, do
     p.lambda = lambda;
     p.coef = h->coef;
     p.result = h->result;
+    p.error_word = h->error_word;
     {
         KernelTimer t(h, st, QN_TIME_SOLVE);
         if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) return QN_ERR_CUDA;
@@ -213,6 +216,8 @@ extern "C" qn_status qn_create(int64_t n, int32_t m, qn_dtype dtype, qn_handle* 
     ok = ok && cudaMalloc(&h->result, sizeof(qn_result_block)) == cudaSuccess;
     ok = ok && cudaMalloc(&h->raw_gram, sizeof(double) * m * m) == cudaSuccess;
     ok = ok && cudaMalloc(&h->ticket, sizeof(unsigned int)) == cudaSuccess;
+    ok = ok && cudaMalloc(&h->error_word, sizeof(int)) == cudaSuccess;
+    ok = ok && cudaMemset(h->error_word, 0, sizeof(int)) == cudaSuccess;
     ok = ok && cudaMallocHost(&h->host_result, sizeof(qn_result_block)) == cudaSuccess;
     ok = ok && cudaMemset(h->ticket, 0, sizeof(unsigned int)) == cudaSuccess;
     ok = ok && cudaMemset(h->result, 0, sizeof(qn_result_block)) == cudaSuccess;
@@ -235,6 +240,7 @@ extern "C" qn_status qn_destroy(qn_handle h) {
     cudaFree(h->result);
     cudaFree(h->raw_gram);
     cudaFree(h->ticket);
+    cudaFree(h->error_word);
     cudaFree(h->win_theta);
     cudaFree(h->win_g);
     cudaFree(h->stage_theta);
@@ -278,8 +284,8 @@ extern "C" qn_status qn_gram(qn_handle h, const void* g, double* gram_out, void*
     begin_call(h, st);
     int np = 0;
     qn_status s = QN_OK;
-    if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st, &h->last_launches) !=
-        cudaSuccess)
+    if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st, &h->last_launches,
+                       h->error_word) != cudaSuccess)
         s = QN_ERR_CUDA;
     if (s == QN_OK) {
         qn_solve_params p;
@@ -288,6 +294,7 @@ extern "C" qn_status qn_gram(qn_handle h, const void* g, double* gram_out, void*
         p.source = QN_SRC_PARTIALS;
         p.partials = h->partials;
         p.num_partials = np;
+        p.error_word = h->error_word;
         p.gram_out = gram_out;
         p.gram_only = 1;
         p.lambda = 1.0;

@@ -15,6 +15,8 @@
 //             carry the cancellation of the later m x m centring.
 // Every thread owns fixed columns and fixed output entries, so results are bitwise reproducible for
 // a given grid.
+#include <stdlib.h>
+
 #include "qn_device.cuh"
 
 namespace qn {
@@ -391,13 +393,24 @@ static cudaError_t launch_gram_t(const T* g, int64_t n, int m, bool raw, double*
 
 }  // namespace qn
 
+// QN_GRAM_PATH=alu forces the plain-ALU kernels (for A/B measurements); anything else lets the
+// tensor-core kernel take the cases it covers.
+static bool tc_allowed() {
+    const char* v = getenv("QN_GRAM_PATH");
+    return !(v && v[0] == 'a');
+}
+
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
-                           int* num_partials, int max_partials, cudaStream_t st, int* launches) {
-    cudaError_t e = dtype == QN_F32
-                        ? qn::launch_gram_t(static_cast<const float*>(g), n, m, raw, partials, num_partials,
-                                            max_partials, st)
-                        : qn::launch_gram_t(static_cast<const __nv_bfloat16*>(g), n, m, raw, partials, num_partials,
-                                            max_partials, st);
+                           int* num_partials, int max_partials, cudaStream_t st, int* launches, int* error_word) {
+    cudaError_t e;
+    if (!raw && tc_allowed() && qn_gram_tc_applicable(dtype, g, n, m)) {
+        e = qn_launch_gram_tc(dtype, g, n, m, partials, num_partials, max_partials, error_word, st);
+    } else {
+        e = dtype == QN_F32
+                ? qn::launch_gram_t(static_cast<const float*>(g), n, m, raw, partials, num_partials, max_partials, st)
+                : qn::launch_gram_t(static_cast<const __nv_bfloat16*>(g), n, m, raw, partials, num_partials,
+                                    max_partials, st);
+    }
     if (e == cudaSuccess && launches) *launches += 1;
     return e;
 }

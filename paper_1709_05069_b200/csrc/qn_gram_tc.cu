@@ -1,0 +1,445 @@
+// Tensor-core Gram pass for 9 <= m <= 64 and large n (sm_100a: tcgen05.mma with TMEM accumulators).
+//
+// What it computes is what qn_gram.cu computes (paper, Section 2: the means, the centred columns and
+// G^H G, here in reference-shifted form): per column the fp32 mean r of the m Workers' values,
+// x_k = g_k - r, C' = sum_i x x^T and t = sum_i x r, as one fp64 partial per CTA.
+//
+// Why tensor cores: the Gram needs m(m+1) flops per m loaded elements; at m = 32 that already needs
+// most of the fp32 FMA peak to keep up with HBM, and at m = 64 (bf16) three times that peak.
+//
+// How the precision is kept.  Each shifted value (fp32) is split exactly into hi = bf16(x) and
+// lo = bf16(x - hi), 16 significant bits in all.  A tile holds the rows [hi_0..hi_MP-1, lo_0..lo_MP-1]
+// of 64 columns, K-major with the 128-byte swizzle, and ONE MMA with that tile as both operands gives
+// all four blocks hi hi^T, hi lo^T, lo hi^T, lo lo^T; their sum is the Gram of (hi + lo).  One
+// tcgen05.mma costs the issuing thread about 65 cycles whatever its shape, so every instruction is
+// M = N = 128: for MP = 64 that is one tile, for MP = 32 two tiles (64 rows each) share a stage and
+// the instruction computes both diagonal 64 x 64 blocks at once (the off-diagonal blocks are unused).
+// bf16 x bf16
+// products are exact, but the tensor core adds them to its fp32 accumulator with truncation: measured on
+// B200, a chain of L MMA instructions loses about L * 5e-8 of the accumulated value, nearly but not quite
+// uniformly over the matrix.  Chains are therefore kept short: after kFlush tiles (4*kFlush instructions)
+// the accumulator is drained into fp32 registers with round-to-nearest adds (unbiased), and every 16
+// drains those go to fp64.  Measured effect on sigma for inputs with a singular-value gap: relative
+// error of the retained sigma_k about 1e-6 (chains of 4 instructions) to 5e-6 (16 instructions).
+// t is accumulated by the CUDA cores that build the tiles (fp32 products, fp64 every tile).
+//
+// Structure (one persistent CTA per SM, warp-specialised):
+//   warps 0-3   drain warps: tcgen05.ld their TMEM quadrant (one D row per thread), fold the hi and lo
+//               column halves and add into per-thread fp32 accumulators; fp64 in shared memory every 16
+//               drains; the two row halves are added at the end
+//   warp  4     one lane issues tcgen05.mma / tcgen05.commit
+//   warps 5..   producer warps: 128-bit global loads -> registers -> mean by shuffles -> hi/lo split
+//               -> swizzled st.shared; one K tile (64 columns) per warp at a time, stages double-buffered
+// Stages and accumulator buffers are handed over with mbarriers.  Every wait has an iteration limit:
+// when it runs out the CTA sets an abort flag and an error word, stops waiting, finishes its loops,
+// frees its TMEM and returns; its partial is poisoned with NaN so the solve reports the failure.
+#include "qn_device.cuh"
+
+namespace qn {
+
+// Shape per operand size.  A stage is always 128 rows x 64 columns (16 KB): one tile for MP = 64, two
+// tiles for MP = 32.  A producer warp may run ahead of the MMA warp by at most one use of a stage (an
+// mbarrier parity wait cannot tell phase k from phase k+2); with in-order consumption that holds as
+// long as a warp's next tile lies no more than kStages stages ahead, i.e. kProducers <= kStages*kTilesPerStage.
+template <int MP>
+struct TcShape {
+    static constexpr int kTilesPerStage = MP == 32 ? 2 : 1;
+    static constexpr int kProducers = MP == 32 ? 10 : 7;
+    static constexpr int kStages = MP == 32 ? 10 : 9;
+    static constexpr int kThreads = (4 + 1 + kProducers) * 32;
+};
+
+// Tiles accumulated in TMEM between drains: MP = 32 drains after every tile (chains of 4 instructions);
+// MP = 64 has twice the columns per drain and bf16 inputs are less sensitive, so it drains every 4 tiles
+// (every 2 for fp32 storage).
+template <typename T, int MP>
+struct TcFlush {
+    // in stages: one stage = two tiles (MP = 32, each tile its own accumulator block) or one tile (MP = 64)
+    static constexpr int kStagesPerDrain = MP == 32 ? 1 : (sizeof(T) == 4 ? 2 : 4);
+};
+constexpr int kTcTileCols = 64;       // K extent of one tile: 64 bf16 = one 128-byte swizzled row
+constexpr int kTcWideEvery = 16;      // drains between fp32 -> fp64 flushes
+constexpr uint32_t kTcWaitLimit = 1u << 24;  // polls per wait before giving up (each poll may suspend ~1 us)
+
+template <int MP>
+struct TcSmem {
+    static constexpr int kStages = TcShape<MP>::kStages;
+    static constexpr int kProducers = TcShape<MP>::kProducers;
+    alignas(1024) unsigned char stage[kStages][128 * 128];
+    double acc64[MP * 128];  // [Gram column][D row], fp64 sums of the folded rows
+    double tpart[kProducers][MP];
+    alignas(8) uint64_t full[kStages];
+    uint64_t empty[kStages];
+    uint64_t accfull[2];
+    uint64_t accempty[2];
+    uint32_t tmem_base;
+    int abort;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(done)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+// Bounded wait.  Returns false (and raises the abort flag) when the limit runs out or another thread
+// of the CTA has already given up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
+    if (*abort) return false;
+    for (uint32_t it = 0; it < kTcWaitLimit; ++it) {
+        if (mbar_try(bar, parity)) return true;
+        if ((it & 255u) == 255u && *abort) return false;
+    }
+    *abort = 1;
+    return false;
+}
+
+// K-major, 128-byte swizzle, 8-row groups 1024 bytes apart (the tile built by the producer warps).
+__device__ __forceinline__ uint64_t tc_smem_desc(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;              // leading byte offset: unused for this layout
+    d |= (uint64_t)(1024 >> 4) << 32;    // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;              // descriptor version of sm_100
+    d |= (uint64_t)2 << 61;              // 128-byte swizzle
+    return d;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo_elem, float hi_elem) {
+    uint32_t w;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w) : "f"(hi_elem), "f"(lo_elem));
+    return w;
+}
+
+// 16 consecutive fp32 columns of this thread's TMEM lane into r[0..15]
+#define TC_LD16(r, taddr)                                                                                      \
+    asm volatile(                                                                                              \
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "                                                              \
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"                                      \
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),    \
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]) \
+        : "r"(taddr)                                                                                           \
+        : "memory")
+
+template <typename T, int MP>
+__global__ void __launch_bounds__(TcShape<MP>::kThreads, 1)
+gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ partials, int* __restrict__ error_word) {
+    using Smem = TcSmem<MP>;
+    constexpr int RT = 2 * MP;                               // operand rows of one tile: hi rows, then lo rows
+    constexpr int U = TcShape<MP>::kTilesPerStage;           // tiles sharing a 128-row stage
+    constexpr int kStages = TcShape<MP>::kStages;
+    constexpr int kProducers = TcShape<MP>::kProducers;
+    constexpr int kDrainEvery = TcFlush<T, MP>::kStagesPerDrain;
+    constexpr int LD = sizeof(T) == 2 ? 1 : 2;  // 16-byte loads per 8-column chunk of one row
+    constexpr int RPT = 8 / LD;        // rows per producer thread: 8 loads per work item either way
+    constexpr int RQ = MP / RPT;       // row groups across the lanes of a producer warp
+    constexpr int CH = 32 / RQ;        // 8-column chunks handled side by side
+    constexpr int PASSES = 8 / CH;     // work items per thread per tile
+    constexpr uint32_t kTmemCols = 256;  // two accumulator buffers of 128 fp32 columns
+    static_assert(U * RT == 128, "a stage is 128 operand rows");
+
+    extern __shared__ unsigned char smem_raw[];
+    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    volatile int* abort = &sm.abort;
+
+    // Tiles of 64 columns are dealt round-robin to the CTAs; a CTA's tiles are grouped U per stage, and
+    // the count is padded to a multiple of U with all-zero tiles (they add nothing).
+    const int64_t ntiles = (n + kTcTileCols - 1) / kTcTileCols;
+    const int64_t my_tiles = blockIdx.x < ntiles ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const int64_t my_stages = (my_tiles + U - 1) / U;
+    const int64_t my_tiles_padded = my_stages * U;
+    const int64_t ndrain = (my_stages + kDrainEvery - 1) / kDrainEvery;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&sm.full[s], U);
+            mbar_init(&sm.empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&sm.accfull[b], 1);
+            mbar_init(&sm.accempty[b], 4);
+        }
+        sm.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 4) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
+                     "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = sm.tmem_base;
+
+    if (warp < 4) {
+        // ------------------------------------------------------------------ drain warps
+        // D is 128 x 128 (M = 128: row i in TMEM lane i).  Row r belongs to tile r / RT of the stage and
+        // needs that tile's own RT columns only: D[r][cb + c] (hi columns) + D[r][cb + MP + c] (lo columns).
+        const int row = tid;
+        const uint32_t cb = (uint32_t)((row / RT) * RT);
+        float facc[MP];
+#pragma unroll
+        for (int e = 0; e < MP; ++e) facc[e] = 0.f;
+#pragma unroll 4
+        for (int e = 0; e < MP; ++e) sm.acc64[e * 128 + row] = 0.0;
+        for (int64_t f = 0; f < ndrain; ++f) {
+            const int b = (int)(f & 1);
+            mbar_wait(&sm.accfull[b], (uint32_t)((f >> 1) & 1), abort);
+            __syncwarp();
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+            for (int c0 = 0; c0 < MP; c0 += 16) {
+                uint32_t v[16], u[16];
+                const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(b * 128) + cb + c0;
+                TC_LD16(v, taddr);
+                TC_LD16(u, taddr + MP);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj)
+                    facc[c0 + jj] += __uint_as_float(v[jj]) + __uint_as_float(u[jj]);
+            }
+            // the accumulator buffer is free again as soon as every drain warp has read it
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.accempty[b]);
+            if (((f + 1) % kTcWideEvery) == 0 || f == ndrain - 1) {
+#pragma unroll
+                for (int e = 0; e < MP; ++e) {
+                    sm.acc64[e * 128 + row] += (double)facc[e];
+                    facc[e] = 0.f;
+                }
+            }
+        }
+    } else if (warp == 4) {
+        // ------------------------------------------------------------------ MMA issue
+        if (lane == 0) {
+            // kind::f16, fp32 accumulate, bf16 x bf16, both K-major, N = 128, M = 128
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+            for (int64_t p = 0; p < my_stages; ++p) {
+                const int s = (int)(p % kStages);
+                const int64_t f = p / kDrainEvery;
+                const int b = (int)(f & 1);
+                const bool first = (p % kDrainEvery) == 0;
+                if (first) {
+                    mbar_wait(&sm.accempty[b], (uint32_t)(((f >> 1) & 1) ^ 1), abort);
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                }
+                mbar_wait(&sm.full[s], (uint32_t)((p / kStages) & 1), abort);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t sbase = smem_u32(sm.stage[s]);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(b * 128);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const uint64_t desc = tc_smem_desc(sbase + k * 32);
+                    const uint32_t accumulate = (first && k == 0) ? 0u : 1u;
+                    asm volatile(
+                        "{\n .reg .pred p;\n setp.ne.u32 p, %4, 0;\n"
+                        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(d_tmem),
+                        "l"(desc), "l"(desc), "r"(idesc), "r"(accumulate)
+                        : "memory");
+                }
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                                 smem_u32(&sm.empty[s]))
+                             : "memory");
+                if ((p % kDrainEvery) == kDrainEvery - 1 || p == my_stages - 1)
+                    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                                     smem_u32(&sm.accfull[b]))
+                                 : "memory");
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ producer warps
+        // Work item = RPT rows x 8 columns per thread (8 sixteen-byte loads): the warp's lanes are CH
+        // column chunks x RQ row groups, a tile takes PASSES items.  The loads of the next item are
+        // issued before the current one is processed, so a warp always has loads in flight.
+        const int pw = warp - 5;
+        const int rq = lane / CH, cl = lane % CH;
+        const int row0 = rq * RPT;
+        // bf16, MP = 64: two row groups share a quarter-warp; the odd one walks its rows in the order
+        // 4,5,6,7,0,1,2,3 so that the two groups' 16-byte stores land on different swizzle positions.
+        const int sw = (RPT == 8 && CH == 4) ? ((rq & 1) << 2) : 0;
+        const float inv_m = 1.0f / (float)m;
+        float tacc[RPT];
+        double tacc64[RPT];
+#pragma unroll
+        for (int j = 0; j < RPT; ++j) {
+            tacc[j] = 0.f;
+            tacc64[j] = 0.0;
+        }
+        auto issue_loads = [&](uint4 (&raw)[RPT][LD], int64_t q, int pass) {
+            const int64_t i0 = (blockIdx.x + q * (int64_t)gridDim.x) * kTcTileCols + (cl + CH * pass) * 8;
+#pragma unroll
+            for (int j = 0; j < RPT; ++j) {
+#pragma unroll
+                for (int l = 0; l < LD; ++l) {
+                    raw[j][l] = make_uint4(0, 0, 0, 0);
+                    const int64_t i = i0 + l * (8 / LD);
+                    const int row = row0 + (j ^ sw);
+                    if (q < my_tiles && row < m && i < n) raw[j][l] = ldg_stream16(g + (int64_t)row * n + i);
+                }
+            }
+        };
+        uint4 nxt[RPT][LD];
+        issue_loads(nxt, pw, 0);
+        for (int64_t q = pw; q < my_tiles_padded; q += kProducers) {
+            const int64_t p = q / U;                 // stage use this tile belongs to
+            const int s = (int)(p % kStages);
+            unsigned char* tile = sm.stage[s] + (int)(q % U) * (RT * 128);
+#pragma unroll
+            for (int pass = 0; pass < PASSES; ++pass) {
+                const int c = cl + CH * pass;
+                uint4 raw[RPT][LD];
+#pragma unroll
+                for (int j = 0; j < RPT; ++j)
+#pragma unroll
+                    for (int l = 0; l < LD; ++l) raw[j][l] = nxt[j][l];
+                if (pass + 1 < PASSES)
+                    issue_loads(nxt, q, pass + 1);
+                else
+                    issue_loads(nxt, q + kProducers, 0);
+                // column sums over this thread's rows, then over the RQ row groups of the warp
+                float r[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    float sum = 0.f;
+#pragma unroll
+                    for (int j = 0; j < RPT; ++j) sum += Storage<T>::get(raw[j][e / (8 / LD)], e % (8 / LD));
+                    r[e] = sum;
+                }
+#pragma unroll
+                for (int o = CH; o < 32; o <<= 1) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) r[e] += __shfl_xor_sync(0xffffffffu, r[e], o);
+                }
+#pragma unroll
+                for (int e = 0; e < 8; ++e) r[e] *= inv_m;
+                if (pass == 0)  // the stage must have been consumed by the MMAs of its previous use
+                    mbar_wait(&sm.empty[s], (uint32_t)(((p / kStages) & 1) ^ 1), abort);
+#pragma unroll
+                for (int j = 0; j < RPT; ++j) {
+                    const int row = row0 + (j ^ sw);
+                    const bool real = row < m;
+                    float x[8], lo[8];
+                    uint32_t hw[4], lw[4];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const float v = Storage<T>::get(raw[j][e / (8 / LD)], e % (8 / LD));
+                        x[e] = real ? v - r[e] : 0.f;
+                        tacc[j] = fmaf(x[e], r[e], tacc[j]);
+                    }
+#pragma unroll
+                    for (int pp = 0; pp < 4; ++pp) {
+                        hw[pp] = pack_bf16x2_rn(x[2 * pp], x[2 * pp + 1]);
+                        lo[2 * pp] = x[2 * pp] - __uint_as_float(hw[pp] << 16);
+                        lo[2 * pp + 1] = x[2 * pp + 1] - __uint_as_float(hw[pp] & 0xffff0000u);
+                        lw[pp] = pack_bf16x2_rn(lo[2 * pp], lo[2 * pp + 1]);
+                    }
+                    // operand row `row` (hi) and MP + row (lo); both have the same row & 7
+                    const uint32_t off = (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4));
+                    *reinterpret_cast<uint4*>(tile + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                    *reinterpret_cast<uint4*>(tile + MP * 128 + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < RPT; ++j) {
+                tacc64[j] += (double)tacc[j];
+                tacc[j] = 0.f;
+            }
+            // make the generic-proxy stores visible to the tensor core, then hand the tile over
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.full[s]);
+        }
+        // t of this warp: add the CH lanes that share a row group (fixed butterfly order)
+#pragma unroll
+        for (int j = 0; j < RPT; ++j) {
+            double v = tacc64[j];
+#pragma unroll
+            for (int o = 1; o < CH; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            if (cl == 0) sm.tpart[pw][row0 + (j ^ sw)] = v;
+        }
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    const double qnan = __longlong_as_double(0x7ff8000000000000ll);
+    const bool poisoned = *abort != 0;
+    double* out = partials + (int64_t)blockIdx.x * qn_partial_len(m);
+    if (tid < 128) {
+        // C'[a][bc]: hi rows and lo rows of the folded accumulators, over the U tiles of a stage
+        constexpr int PER = MP * MP / 128;
+        const int a = tid % MP, h = tid / MP;
+#pragma unroll 4
+        for (int e = 0; e < PER; ++e) {
+            const int bc = h * PER + e;
+            if (a <= bc && bc < m) {
+                double v = 0.0;
+#pragma unroll
+                for (int u = 0; u < U; ++u) v += sm.acc64[bc * 128 + u * RT + a] + sm.acc64[bc * 128 + u * RT + MP + a];
+                out[qn_tri_index(m, a, bc)] = poisoned ? qnan : v;
+            }
+        }
+    }
+    if (tid < m) {
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < kProducers; ++w) s += sm.tpart[w][tid];
+        out[m * (m + 1) / 2 + tid] = poisoned ? qnan : s;
+    }
+    if (tid == 0 && *abort && error_word) atomicExch(error_word, 1);
+    if (warp == 4) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+template <typename T, int MP>
+static cudaError_t launch_tc(const T* g, int64_t n, int m, double* partials, int grid, int* error_word,
+                             cudaStream_t st) {
+    auto kern = gram_tc_kernel<T, MP>;
+    const size_t smem = sizeof(TcSmem<MP>) + 1024;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, TcShape<MP>::kThreads, smem, st>>>(g, n, m, partials, error_word);
+    return cudaGetLastError();
+}
+
+}  // namespace qn
+
+bool qn_gram_tc_applicable(qn_dtype dtype, const void* g, int64_t n, int m) {
+    const int64_t elem = dtype == QN_F32 ? 4 : 2;
+    return m > 8 && m <= QN_MAX_M && n >= QN_PRECISE_BELOW && (reinterpret_cast<uintptr_t>(g) % 16 == 0) &&
+           ((n * elem) % 16 == 0);
+}
+
+cudaError_t qn_launch_gram_tc(qn_dtype dtype, const void* g, int64_t n, int m, double* partials, int* num_partials,
+                              int max_partials, int* error_word, cudaStream_t st) {
+    const int sms = qn_sm_count();
+    const int64_t ntiles = (n + qn::kTcTileCols - 1) / qn::kTcTileCols;
+    int grid = (int)(ntiles < sms ? ntiles : sms);
+    if (grid > max_partials) grid = max_partials;
+    *num_partials = grid;
+    if (dtype == QN_F32) {
+        const float* p = static_cast<const float*>(g);
+        return m <= 32 ? qn::launch_tc<float, 32>(p, n, m, partials, grid, error_word, st)
+                       : qn::launch_tc<float, 64>(p, n, m, partials, grid, error_word, st);
+    }
+    const __nv_bfloat16* p = static_cast<const __nv_bfloat16*>(g);
+    return m <= 32 ? qn::launch_tc<__nv_bfloat16, 32>(p, n, m, partials, grid, error_word, st)
+                   : qn::launch_tc<__nv_bfloat16, 64>(p, n, m, partials, grid, error_word, st);
+}

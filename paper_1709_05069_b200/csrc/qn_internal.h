@@ -58,11 +58,17 @@ struct qn_solve_params {
     double tau, lambda;
     qn_coef_block* coef;
     qn_result_block* result;
+    int* error_word;      // device int set by a kernel that gave up on a bounded wait (may be NULL); read and cleared
 };
 
 // Launchers.  Each returns the launch error and adds the kernels it launched to *launches.
+// error_word (device int, may be NULL) is set to 1 by a kernel that gave up on a bounded wait.
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
-                           int* num_partials, int max_partials, cudaStream_t st, int* launches);
+                           int* num_partials, int max_partials, cudaStream_t st, int* launches,
+                           int* error_word = nullptr);
+bool qn_gram_tc_applicable(qn_dtype dtype, const void* g, int64_t n, int m);
+cudaError_t qn_launch_gram_tc(qn_dtype dtype, const void* g, int64_t n, int m, double* partials, int* num_partials,
+                              int max_partials, int* error_word, cudaStream_t st);
 cudaError_t qn_launch_solve(const qn_solve_params& p, cudaStream_t st, int* launches);
 cudaError_t qn_launch_combine(qn_dtype dtype, const void* theta, const void* g, int64_t n, int m,
                               const qn_coef_block* coef, void* theta_new, cudaStream_t st, int* launches);

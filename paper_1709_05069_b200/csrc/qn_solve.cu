@@ -34,6 +34,7 @@ struct SolveSmem {
     int order[QN_MAX_M];
     int flag_nonfinite;
     int flag_rotated;
+    int flag_timeout;
     int j;
 };
 
@@ -75,6 +76,11 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
         sm.flag_nonfinite = 0;
         sm.flag_rotated = 0;
         sm.j = 0;
+        sm.flag_timeout = 0;
+        if (prm.error_word && *prm.error_word) {  // a streaming kernel gave up on a wait: report and clear
+            sm.flag_timeout = 1;
+            *prm.error_word = 0;
+        }
     }
     // ---------------------------------------------------------------- phase 1: C' and t
     if (prm.source == QN_SRC_PARTIALS) {
@@ -142,7 +148,7 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
     __syncthreads();
     if (prm.gram_only) {
         if (tid == 0 && prm.result) {
-            prm.result->status = sm.flag_nonfinite ? QN_ERR_NONFINITE : QN_OK;
+            prm.result->status = sm.flag_timeout ? QN_ERR_DEVICE_TIMEOUT : sm.flag_nonfinite ? QN_ERR_NONFINITE : QN_OK;
             prm.result->j = 0;
             prm.result->sweeps = 0;
         }
@@ -158,7 +164,7 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
             prm.coef->inv_m = (float)inv_m;
             prm.coef->m = m;
             prm.result->j = 0;
-            prm.result->status = QN_ERR_NONFINITE;
+            prm.result->status = sm.flag_timeout ? QN_ERR_DEVICE_TIMEOUT : QN_ERR_NONFINITE;
             prm.result->sweeps = 0;
         }
         return;
@@ -302,7 +308,7 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
         prm.coef->inv_m = (float)inv_m;
         prm.coef->m = m;
         prm.result->j = j;
-        prm.result->status = converged ? QN_OK : QN_ERR_NOT_CONVERGED;
+        prm.result->status = sm.flag_timeout ? QN_ERR_DEVICE_TIMEOUT : converged ? QN_OK : QN_ERR_NOT_CONVERGED;
         prm.result->sweeps = sweeps;
     }
 }

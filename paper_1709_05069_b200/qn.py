@@ -15,7 +15,8 @@ QN_F32 = 0
 QN_BF16 = 1
 QN_MAX_M = 64
 
-QN_OK, QN_ERR_INVALID, QN_ERR_ALLOC, QN_ERR_CUDA, QN_ERR_STATE, QN_ERR_NOT_CONVERGED, QN_ERR_NONFINITE = range(7)
+(QN_OK, QN_ERR_INVALID, QN_ERR_ALLOC, QN_ERR_CUDA, QN_ERR_STATE, QN_ERR_NOT_CONVERGED, QN_ERR_NONFINITE,
+ QN_ERR_DEVICE_TIMEOUT) = range(8)
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libqn.so")
 _lib: Optional[ctypes.CDLL] = None

@@ -31,8 +31,8 @@ def test_exports_every_declared_symbol(qn):
 
 
 def test_strerror(qn):
-    texts = {qn.qn_strerror(s) for s in range(7)}
-    assert len(texts) == 7 and "ok" in texts
+    texts = {qn.qn_strerror(s) for s in range(8)}
+    assert len(texts) == 8 and "ok" in texts
     assert qn.qn_strerror(99) == "unknown status"
 
 
