@@ -49,13 +49,13 @@ struct TcShape {
     static constexpr int kThreads = (4 + 1 + kProducers) * 32;
 };
 
-// Tiles accumulated in TMEM between drains: MP = 32 drains after every tile (chains of 4 instructions);
-// MP = 64 has twice the columns per drain and bf16 inputs are less sensitive, so it drains every 4 tiles
-// (every 2 for fp32 storage).
+// Stages accumulated in TMEM between drains.  A drain's TMEM loads queue behind the MMAs already issued,
+// so very frequent drains stall the MMA thread; very long chains lose accuracy (see the header).  MP = 32:
+// every 2 stages (each tile's block then sees chains of 8 instructions); MP = 64: every 4 stages for bf16
+// storage, every 2 for fp32 storage, whose inputs carry more bits below the hi/lo split.
 template <typename T, int MP>
 struct TcFlush {
-    // in stages: one stage = two tiles (MP = 32, each tile its own accumulator block) or one tile (MP = 64)
-    static constexpr int kStagesPerDrain = MP == 32 ? 1 : (sizeof(T) == 4 ? 2 : 4);
+    static constexpr int kStagesPerDrain = MP == 32 ? 2 : (sizeof(T) == 4 ? 2 : 4);
 };
 constexpr int kTcTileCols = 64;       // K extent of one tile: 64 bf16 = one 128-byte swizzled row
 constexpr int kTcWideEvery = 16;      // drains between fp32 -> fp64 flushes
@@ -70,8 +70,8 @@ struct TcSmem {
     double tpart[kProducers][MP];
     alignas(8) uint64_t full[kStages];
     uint64_t empty[kStages];
-    uint64_t accfull[2];
-    uint64_t accempty[2];
+    uint64_t accfull[4];
+    uint64_t accempty[4];
     uint32_t tmem_base;
     int abort;
 };
@@ -96,6 +96,7 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
 // Bounded wait.  Returns false (and raises the abort flag) when the limit runs out or another thread
 // of the CTA has already given up.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
+    if (mbar_try(bar, parity)) return true;  // the common case costs one shared-memory round trip
     if (*abort) return false;
     for (uint32_t it = 0; it < kTcWaitLimit; ++it) {
         if (mbar_try(bar, parity)) return true;
@@ -146,7 +147,8 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
     constexpr int RQ = MP / RPT;       // row groups across the lanes of a producer warp
     constexpr int CH = 32 / RQ;        // 8-column chunks handled side by side
     constexpr int PASSES = 8 / CH;     // work items per thread per tile
-    constexpr uint32_t kTmemCols = 256;  // two accumulator buffers of 128 fp32 columns
+    constexpr uint32_t kTmemCols = 512;  // four accumulator buffers of 128 fp32 columns: all of TMEM
+    constexpr int kAccBufs = 4;
     static_assert(U * RT == 128, "a stage is 128 operand rows");
 
     extern __shared__ unsigned char smem_raw[];
@@ -167,7 +169,7 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
             mbar_init(&sm.full[s], U);
             mbar_init(&sm.empty[s], 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < kAccBufs; ++b) {
             mbar_init(&sm.accfull[b], 1);
             mbar_init(&sm.accempty[b], 4);
         }
@@ -196,27 +198,39 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
         for (int e = 0; e < MP; ++e) facc[e] = 0.f;
 #pragma unroll 4
         for (int e = 0; e < MP; ++e) sm.acc64[e * 128 + row] = 0.0;
-        for (int64_t f = 0; f < ndrain; ++f) {
-            const int b = (int)(f & 1);
-            mbar_wait(&sm.accfull[b], (uint32_t)((f >> 1) & 1), abort);
+        const int ndrains = (int)ndrain;
+        int b = 0, since_wide = 0;
+        uint32_t acc_par = 0;
+        for (int f = 0; f < ndrains; ++f) {
+            mbar_wait(&sm.accfull[b], acc_par, abort);
             __syncwarp();
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            // 32 Gram columns per round: hi and lo halves, four 16-column loads in flight, one wait
 #pragma unroll
-            for (int c0 = 0; c0 < MP; c0 += 16) {
-                uint32_t v[16], u[16];
+            for (int c0 = 0; c0 < MP; c0 += 32) {
+                uint32_t v0[16], v1[16], u0[16], u1[16];
                 const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(b * 128) + cb + c0;
-                TC_LD16(v, taddr);
-                TC_LD16(u, taddr + MP);
+                TC_LD16(v0, taddr);
+                TC_LD16(v1, taddr + 16);
+                TC_LD16(u0, taddr + MP);
+                TC_LD16(u1, taddr + MP + 16);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-                for (int jj = 0; jj < 16; ++jj)
-                    facc[c0 + jj] += __uint_as_float(v[jj]) + __uint_as_float(u[jj]);
+                for (int jj = 0; jj < 16; ++jj) {
+                    facc[c0 + jj] += __uint_as_float(v0[jj]) + __uint_as_float(u0[jj]);
+                    facc[c0 + 16 + jj] += __uint_as_float(v1[jj]) + __uint_as_float(u1[jj]);
+                }
             }
             // the accumulator buffer is free again as soon as every drain warp has read it
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.accempty[b]);
-            if (((f + 1) % kTcWideEvery) == 0 || f == ndrain - 1) {
+            if (++b == kAccBufs) {
+                b = 0;
+                acc_par ^= 1u;
+            }
+            if (++since_wide == kTcWideEvery || f == ndrains - 1) {
+                since_wide = 0;
 #pragma unroll
                 for (int e = 0; e < MP; ++e) {
                     sm.acc64[e * 128 + row] += (double)facc[e];
@@ -229,36 +243,49 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
         if (lane == 0) {
             // kind::f16, fp32 accumulate, bf16 x bf16, both K-major, N = 128, M = 128
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-            for (int64_t p = 0; p < my_stages; ++p) {
-                const int s = (int)(p % kStages);
-                const int64_t f = p / kDrainEvery;
-                const int b = (int)(f & 1);
-                const bool first = (p % kDrainEvery) == 0;
+            // One thread runs this loop and every instruction in it is on the critical path of the whole
+            // CTA, so stage index, parities and descriptors are carried along instead of recomputed.
+            const uint64_t desc0 = tc_smem_desc(smem_u32(sm.stage[0]));
+            const int nstages = (int)my_stages;
+            int s = 0, b = 0, in_chain = 0;
+            uint32_t full_par = 0, acc_par = 0;
+            for (int p = 0; p < nstages; ++p) {
+                const bool first = in_chain == 0;
                 if (first) {
-                    mbar_wait(&sm.accempty[b], (uint32_t)(((f >> 1) & 1) ^ 1), abort);
+                    mbar_wait(&sm.accempty[b], acc_par ^ 1u, abort);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 }
-                mbar_wait(&sm.full[s], (uint32_t)((p / kStages) & 1), abort);
+                mbar_wait(&sm.full[s], full_par, abort);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t sbase = smem_u32(sm.stage[s]);
+                // the start-address field counts 16-byte units: a stage is 16 KB, a K step of 16 bf16 is 32 B
+                const uint64_t desc = desc0 + (uint64_t)(s * (16384 >> 4));
                 const uint32_t d_tmem = tmem_base + (uint32_t)(b * 128);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    const uint64_t desc = tc_smem_desc(sbase + k * 32);
                     const uint32_t accumulate = (first && k == 0) ? 0u : 1u;
                     asm volatile(
                         "{\n .reg .pred p;\n setp.ne.u32 p, %4, 0;\n"
                         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(d_tmem),
-                        "l"(desc), "l"(desc), "r"(idesc), "r"(accumulate)
+                        "l"(desc + 2 * k), "l"(desc + 2 * k), "r"(idesc), "r"(accumulate)
                         : "memory");
                 }
                 asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
                                  smem_u32(&sm.empty[s]))
                              : "memory");
-                if ((p % kDrainEvery) == kDrainEvery - 1 || p == my_stages - 1)
+                if (++in_chain == kDrainEvery || p == nstages - 1) {
                     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
                                      smem_u32(&sm.accfull[b]))
                                  : "memory");
+                    in_chain = 0;
+                    if (++b == kAccBufs) {
+                        b = 0;
+                        acc_par ^= 1u;
+                    }
+                }
+                if (++s == kStages) {
+                    s = 0;
+                    full_par ^= 1u;
+                }
             }
         }
         __syncwarp();

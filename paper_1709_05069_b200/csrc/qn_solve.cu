@@ -188,6 +188,7 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
     }
     fro = sqrt(block_sum(fro, sm.red));
     const double thresh = 1e-15 * fro;
+    const double inv_fro = fro > 0.0 ? 1.0 / fro : 0.0;  // brings entries into fp32 range whatever the data's scale
     const int pa_idx = tid / H, pb_idx = tid % H;
     const bool worker = tid < H * H;
     int sweeps = 0;
@@ -202,10 +203,19 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
                     const double apq = sm.A[pa * kLd + qa];
                     double c = 1.0, s = 0.0, t = 0.0;
                     if (fabs(apq) > thresh) {
+                        // tan of the rotation angle from fp32 arithmetic (relative error ~1e-7): the
+                        // rotation then leaves a'_pq = O(1e-7 a_pq) instead of 0, which the next sweep
+                        // removes; what must hold to fp64 accuracy is c^2 + s^2 = 1, and c = rsqrt(1 + t^2)
+                        // is refined to full precision by two Newton steps.
                         const double app = sm.A[pa * kLd + pa], aqq = sm.A[qa * kLd + qa];
-                        const double zeta = (aqq - app) / (2.0 * apq);
-                        t = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
-                        c = 1.0 / sqrt(1.0 + t * t);
+                        const float zeta = (float)((aqq - app) * inv_fro) / (2.0f * (float)(apq * inv_fro));
+                        const float tf = copysignf(1.0f, zeta) / (fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.0f)));
+                        t = (double)tf;
+                        const double x = fma(t, t, 1.0);
+                        double y = (double)rsqrtf((float)x);
+                        y = y * fma(-0.5 * x, y * y, 1.5);
+                        y = y * fma(-0.5 * x, y * y, 1.5);
+                        c = y;
                         s = t * c;
                         sm.flag_rotated = 1;
                     }
@@ -221,18 +231,14 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
                 const double x00 = sm.A[pa * kLd + pb], x01 = sm.A[pa * kLd + qb];
                 const double x10 = sm.A[qa * kLd + pb], x11 = sm.A[qa * kLd + qb];
                 double y00, y01, y10, y11;
-                if (pa_idx == pb_idx) {
-                    const double t = sm.rot_t[pa_idx];
-                    y00 = x00 - t * x01;
-                    y11 = x11 + t * x01;
-                    y01 = y10 = (sa == 0.0 && ca == 1.0) ? x01 : 0.0;  // untouched if the rotation was skipped
-                } else {
+                {
                     const double t00 = cb * x00 - sb * x01, t01 = sb * x00 + cb * x01;
                     const double t10 = cb * x10 - sb * x11, t11 = sb * x10 + cb * x11;
                     y00 = ca * t00 - sa * t10;
                     y10 = sa * t00 + ca * t10;
                     y01 = ca * t01 - sa * t11;
                     y11 = sa * t01 + ca * t11;
+                    if (pa_idx == pb_idx) y01 = y10 = 0.5 * (y01 + y10);  // keep the matrix exactly symmetric
                 }
                 sm.A[pa * kLd + pb] = y00;
                 sm.A[pa * kLd + qb] = y01;
