@@ -346,3 +346,95 @@ def test_argument_validation(qn):
     assert L.qn_update_window(hd.ptr, 1.0, 0.1, o.data_ptr(), None, None, st) == qn.QN_ERR_STATE
     assert L.qn_status_sync(hd.ptr) == qn.QN_OK
     hd.close()
+
+
+# --------------------------------------------------------------------------- tensor-core Gram path (n >= 2^22, m > 8)
+@pytest.mark.parametrize("dtype,m,n,gap", [
+    ("f32", 32, (1 << 22) + 64 * 3 + 4, True),     # config 2's shape class: two tiles per stage, ragged tail
+    ("f32", 9, 1 << 22, True),                     # smallest m on this path: 23 padding rows
+    ("f32", 33, 1 << 22, True),                    # first m with one tile per stage
+    ("bf16", 16, (1 << 22) + 8 * 13, True),
+    ("bf16", 64, 1 << 22, True),                   # config 4's shape class
+    ("bf16", 64, 1 << 22, False),
+])
+def test_tensor_core_gram_path(qn, dtype, m, n, gap):
+    """Above 2^22 columns and 8 Workers the Gram pass runs on the tensor cores (bf16 hi/lo split, fp32
+    accumulation in short chains).  Same bar as everywhere: exact j, sigma and theta_new tolerances."""
+    import os
+
+    assert os.environ.get("QN_GRAM_PATH", "") != "alu"
+    cfg = W.Config(40, n, m, dtype, -2, 2, 0, 0.01, 1e-4, 1.0, 0.01)
+    lam = 0.05 if (gap and dtype == "bf16") else 0.01
+    theta, g = W.generate(cfg, "cuda", gap_lam=lam if gap else None, gap_scale=1.0 if (gap and dtype == "bf16") else None)
+    expect = assert_gap(theta, g, lam) if gap else m - 1
+    check_against_oracle(qn, theta, g, cfg.tau, lam, dtype, expect_j=expect)
+
+
+def test_tensor_core_and_alu_paths_agree(qn):
+    """The same input through the tensor-core kernel and (QN_GRAM_PATH=alu) the plain-ALU kernel."""
+    import os
+
+    cfg = W.Config(41, 1 << 22, 24, "f32", -2, 2, 0, 0.01, 1e-4, 1.0, 0.01)
+    theta, g = W.generate(cfg, "cuda", gap_lam=0.01)
+    out = {}
+    for path in ("tc", "alu"):
+        os.environ["QN_GRAM_PATH"] = path
+        try:
+            out[path] = run_gpu(qn, theta, g, cfg.tau, cfg.lam)
+        finally:
+            os.environ.pop("QN_GRAM_PATH", None)
+    (o1, j1, s1, st1, _), (o2, j2, s2, st2, _) = out["tc"], out["alu"]
+    assert st1 == 0 and st2 == 0 and j1 == j2
+    assert np.max(np.abs(s1[:j1] - s2[:j1]) / s2[:j1]) <= 1e-5
+    assert torch.linalg.norm(o1.double() - o2.double()) / torch.linalg.norm(o2.double()) <= 1e-5
+
+
+def test_tensor_core_path_bitwise_reproducible(qn):
+    cfg = W.Config(42, (1 << 22) + 640, 32, "f32", -2, 2, 0, 0.01, 1e-4, 1.0, 0.01)
+    theta, g = W.generate(cfg, "cuda")
+    a, ja, sa, _, _ = run_gpu(qn, theta, g, 0.5, 0.01)
+    b, jb, sb, _, _ = run_gpu(qn, theta, g, 0.5, 0.01)
+    assert ja == jb and np.array_equal(sa, sb) and torch.equal(a.view(torch.int32), b.view(torch.int32))
+
+
+# --------------------------------------------------------------------------- full size, in the benchmark's launch configuration
+def test_config2_full_size_sampled(qn):
+    """Config 2 at its full n = 25.6 M, m = 32, fp32, exactly as bench.py launches it: j and sigma from the
+    oracle's full passes over the same bits, theta_new on 4096 sampled columns (first, last, tile edges, random)."""
+    cfg = W.CONFIGS[2]
+    theta, g = W.generate(cfg, "cuda")
+    rng = np.random.default_rng(7)
+    idx = np.unique(np.concatenate([[0, 1, 63, 64, 127, 128, cfg.n - 1, cfg.n - 64, cfg.n - 65],
+                                    rng.integers(0, cfg.n, 4096)])).astype(np.int64)
+    rel, j, _ = check_against_oracle(qn, theta, g, cfg.tau, cfg.lam, cfg.dtype, expect_j=cfg.m - 1, sample=idx)
+    assert j == cfg.m - 1
+
+
+def test_config4_full_size_by_tiling(qn):
+    """Config 4 at its full n = 2^28, m = 64, bf16 (68.7 GB of inputs) is beyond what the oracle can read in a
+    test.  Property used instead: if the columns repeat with period p, the Gram is (n/p) times the block's Gram,
+    so sigma scales by sqrt(n/p), j is unchanged and theta_new repeats with the block's values.  The block
+    (p = 2^18 columns) goes through the oracle; the full-size input goes through the library."""
+    free, _ = torch.cuda.mem_get_info()
+    cfg = W.CONFIGS[4]
+    need = 2 * cfg.m * cfg.n * 2 + cfg.n * 2 + (2 << 30)
+    if free < need:
+        pytest.skip("needs %.0f GB of free device memory" % (need / 1e9))
+    p = 1 << 18
+    block = cfg.with_shape(n=p)
+    tb, gb = W.generate(block, "cuda")
+    theta = W.tile_columns(tb, cfg.n)
+    g = W.tile_columns(gb, cfg.n)
+    out, j, sigma, status, launches = run_gpu(qn, theta, g, cfg.tau, cfg.lam)
+    del theta, g
+    ref = oracle.update(W.to_bits(tb), W.to_bits(gb), cfg.tau, cfg.lam)
+    assert status == 0 and launches == 3 and j == ref.j == cfg.m - 1
+    scale = np.sqrt(cfg.n / p)
+    assert np.max(np.abs(sigma - scale * ref.sigma)) <= 1e-5 * scale * ref.sigma[0]
+    assert np.max(np.abs(sigma[:j] - scale * ref.sigma[:j]) / (scale * ref.sigma[:j])) <= 1e-5
+    got = oracle.storage_to_f64(W.to_bits(out))
+    for start in (0, p, 7 * p, cfg.n - p):
+        seg = got[start:start + p]
+        assert np.linalg.norm(seg - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL["bf16"]
+    # every period holds the same bits
+    assert torch.equal(out[:p].view(torch.int16), out[cfg.n - p:].view(torch.int16))
