@@ -53,6 +53,13 @@ __device__ __forceinline__ uint4 ldg_stream16(const void* p) {
     return v;
 }
 
+// 32-byte read-only load (one full sector per request; the address must be 32-byte aligned).
+__device__ __forceinline__ void ldg_stream32(const void* p, uint4& a, uint4& b) {
+    asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w), "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w)
+                 : "l"(p));
+}
+
 // 16-byte streaming store (written once, not re-read by this kernel).
 __device__ __forceinline__ void stg_stream16(void* p, const uint4& v) {
     asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)

@@ -312,12 +312,16 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
             const int64_t i0 = (blockIdx.x + q * (int64_t)gridDim.x) * kTcTileCols + (cl + CH * pass) * 8;
 #pragma unroll
             for (int j = 0; j < RPT; ++j) {
+                const int row = row0 + (j ^ sw);
 #pragma unroll
-                for (int l = 0; l < LD; ++l) {
-                    raw[j][l] = make_uint4(0, 0, 0, 0);
-                    const int64_t i = i0 + l * (8 / LD);
-                    const int row = row0 + (j ^ sw);
-                    if (q < my_tiles && row < m && i < n) raw[j][l] = ldg_stream16(g + (int64_t)row * n + i);
+                for (int l = 0; l < LD; ++l) raw[j][l] = make_uint4(0, 0, 0, 0);
+                if (q < my_tiles && row < m && i0 < n) {
+                    // rows are 32-byte aligned and n is a multiple of 8 on this path (see
+                    // qn_gram_tc_applicable), so an 8-column chunk is never cut by the end of the row
+                    if (LD == 1)
+                        raw[j][0] = ldg_stream16(g + (int64_t)row * n + i0);
+                    else
+                        ldg_stream32(g + (int64_t)row * n + i0, raw[j][0], raw[j][LD - 1]);
                 }
             }
         };
@@ -450,8 +454,10 @@ static cudaError_t launch_tc(const T* g, int64_t n, int m, double* partials, int
 
 bool qn_gram_tc_applicable(qn_dtype dtype, const void* g, int64_t n, int m) {
     const int64_t elem = dtype == QN_F32 ? 4 : 2;
-    return m > 8 && m <= QN_MAX_M && n >= QN_PRECISE_BELOW && (reinterpret_cast<uintptr_t>(g) % 16 == 0) &&
-           ((n * elem) % 16 == 0);
+    // every 8-column chunk of a row is fetched with one load: 16 bytes (bf16) or 32 bytes (fp32), aligned
+    const int64_t chunk = 8 * elem;
+    return m > 8 && m <= QN_MAX_M && n >= QN_PRECISE_BELOW && (reinterpret_cast<uintptr_t>(g) % chunk == 0) &&
+           (n % 8 == 0);
 }
 
 cudaError_t qn_launch_gram_tc(qn_dtype dtype, const void* g, int64_t n, int m, double* partials, int* num_partials,
