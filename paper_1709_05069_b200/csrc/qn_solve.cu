@@ -171,8 +171,15 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
     }
 
     // ---------------------------------------------------------------- phase 3: two-sided Jacobi
+    // Round-robin ordering: M2/2 disjoint pairs per round, M2-1 rounds per sweep.  Thread (a, b) owns
+    // the 2x2 block (rows of pair a) x (columns of pair b) for the round.  It reads the diagonal blocks
+    // of its two pairs and its own block, everybody synchronises, and it then computes BOTH rotations
+    // itself (the same numbers in every thread that needs them) and writes its block: two barriers per
+    // round and no separate "compute the angles" phase on the critical path.
     const int M2 = m + (m & 1);
     const int H = M2 / 2;
+    const int N = M2 - 1;
+    const int jthreads = H * H > QN_MAX_M ? ((H * H + 31) / 32) * 32 : QN_MAX_M;  // threads that take part from here on
     if (M2 > m) {
         for (int e = tid; e < M2; e += nthr) {
             sm.A[m * kLd + e] = 0.0;
@@ -187,80 +194,103 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
         fro += a * a;
     }
     fro = sqrt(block_sum(fro, sm.red));
+    if (tid >= jthreads) return;  // the remaining phases synchronise with a named barrier over jthreads
     const double thresh = 1e-15 * fro;
     const double inv_fro = fro > 0.0 ? 1.0 / fro : 0.0;  // brings entries into fp32 range whatever the data's scale
     const int pa_idx = tid / H, pb_idx = tid % H;
     const bool worker = tid < H * H;
+    // positions of this thread's two pairs in round 0; each round both members move one step round the circle
+    int a0 = pa_idx == 0 ? N : pa_idx % N, a1 = pa_idx == 0 ? 0 : (N - pa_idx) % N;
+    int b0 = pb_idx == 0 ? N : pb_idx % N, b1 = pb_idx == 0 ? 0 : (N - pb_idx) % N;
     int sweeps = 0;
     bool converged = (fro == 0.0) || m < 2;
+    auto rotation = [&](double app, double aqq, double apq, double& c, double& s) {
+        c = 1.0;
+        s = 0.0;
+        if (fabs(apq) > thresh) {
+            // tan of the rotation angle from fp32 arithmetic (relative error ~1e-7): the rotation then
+            // leaves a'_pq = O(1e-7 a_pq) instead of 0, which the next sweep removes.  What must hold to
+            // fp64 accuracy is c^2 + s^2 = 1: c = rsqrt(1 + t^2) is refined by two Newton steps.
+            const float zeta = (float)((aqq - app) * inv_fro) / (2.0f * (float)(apq * inv_fro));
+            const float tf = copysignf(1.0f, zeta) / (fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.0f)));
+            const double t = (double)tf;
+            const double x = fma(t, t, 1.0);
+            double y = (double)rsqrtf((float)x);
+            y = y * fma(-0.5 * x, y * y, 1.5);
+            y = y * fma(-0.5 * x, y * y, 1.5);
+            c = y;
+            s = t * y;
+        }
+    };
     while (!converged && sweeps < kMaxSweeps) {
-        for (int r = 0; r < M2 - 1; ++r) {
-            int pa = 0, qa = 0, pb = 0, qb = 0;
+        for (int r = 0; r < N; ++r) {
+            double ca = 1.0, sa = 0.0, cb = 1.0, sb = 0.0;
+            double x00 = 0, x01 = 0, x10 = 0, x11 = 0, v00 = 0, v01 = 0, v10 = 0, v11 = 0;
+            double daa_pp = 0, daa_qq = 0, daa_pq = 0, dbb_pp = 0, dbb_qq = 0, dbb_pq = 0;
+            const int pa = a0 < a1 ? a0 : a1, qa = a0 < a1 ? a1 : a0;
+            const int pb = b0 < b1 ? b0 : b1, qb = b0 < b1 ? b1 : b0;
             if (worker) {
-                rr_pair(M2, r, pa_idx, pa, qa);
-                rr_pair(M2, r, pb_idx, pb, qb);
-                if (pa_idx == pb_idx) {
-                    const double apq = sm.A[pa * kLd + qa];
-                    double c = 1.0, s = 0.0, t = 0.0;
-                    if (fabs(apq) > thresh) {
-                        // tan of the rotation angle from fp32 arithmetic (relative error ~1e-7): the
-                        // rotation then leaves a'_pq = O(1e-7 a_pq) instead of 0, which the next sweep
-                        // removes; what must hold to fp64 accuracy is c^2 + s^2 = 1, and c = rsqrt(1 + t^2)
-                        // is refined to full precision by two Newton steps.
-                        const double app = sm.A[pa * kLd + pa], aqq = sm.A[qa * kLd + qa];
-                        const float zeta = (float)((aqq - app) * inv_fro) / (2.0f * (float)(apq * inv_fro));
-                        const float tf = copysignf(1.0f, zeta) / (fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.0f)));
-                        t = (double)tf;
-                        const double x = fma(t, t, 1.0);
-                        double y = (double)rsqrtf((float)x);
-                        y = y * fma(-0.5 * x, y * y, 1.5);
-                        y = y * fma(-0.5 * x, y * y, 1.5);
-                        c = y;
-                        s = t * c;
-                        sm.flag_rotated = 1;
-                    }
-                    sm.rot_c[pa_idx] = c;
-                    sm.rot_s[pa_idx] = s;
-                    sm.rot_t[pa_idx] = t;
-                }
+                daa_pp = sm.A[pa * kLd + pa];
+                daa_qq = sm.A[qa * kLd + qa];
+                daa_pq = sm.A[pa * kLd + qa];
+                dbb_pp = sm.A[pb * kLd + pb];
+                dbb_qq = sm.A[qb * kLd + qb];
+                dbb_pq = sm.A[pb * kLd + qb];
+                x00 = sm.A[pa * kLd + pb];
+                x01 = sm.A[pa * kLd + qb];
+                x10 = sm.A[qa * kLd + pb];
+                x11 = sm.A[qa * kLd + qb];
+                v00 = sm.V[(2 * pa_idx) * kLd + pb];
+                v01 = sm.V[(2 * pa_idx) * kLd + qb];
+                v10 = sm.V[(2 * pa_idx + 1) * kLd + pb];
+                v11 = sm.V[(2 * pa_idx + 1) * kLd + qb];
             }
-            __syncthreads();
+            asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");  // all reads done before any write
             if (worker) {
-                const double ca = sm.rot_c[pa_idx], sa = sm.rot_s[pa_idx];
-                const double cb = sm.rot_c[pb_idx], sb = sm.rot_s[pb_idx];
-                const double x00 = sm.A[pa * kLd + pb], x01 = sm.A[pa * kLd + qb];
-                const double x10 = sm.A[qa * kLd + pb], x11 = sm.A[qa * kLd + qb];
-                double y00, y01, y10, y11;
-                {
-                    const double t00 = cb * x00 - sb * x01, t01 = sb * x00 + cb * x01;
-                    const double t10 = cb * x10 - sb * x11, t11 = sb * x10 + cb * x11;
-                    y00 = ca * t00 - sa * t10;
-                    y10 = sa * t00 + ca * t10;
-                    y01 = ca * t01 - sa * t11;
-                    y11 = sa * t01 + ca * t11;
-                    if (pa_idx == pb_idx) y01 = y10 = 0.5 * (y01 + y10);  // keep the matrix exactly symmetric
+                rotation(daa_pp, daa_qq, daa_pq, ca, sa);
+                if (pa_idx == pb_idx) {
+                    cb = ca;
+                    sb = sa;
+                } else {
+                    rotation(dbb_pp, dbb_qq, dbb_pq, cb, sb);
                 }
+                const double t00 = cb * x00 - sb * x01, t01 = sb * x00 + cb * x01;
+                const double t10 = cb * x10 - sb * x11, t11 = sb * x10 + cb * x11;
+                double y00 = ca * t00 - sa * t10, y10 = sa * t00 + ca * t10;
+                double y01 = ca * t01 - sa * t11, y11 = sa * t01 + ca * t11;
+                if (pa_idx == pb_idx) y01 = y10 = 0.5 * (y01 + y10);  // keep the diagonal block symmetric
                 sm.A[pa * kLd + pb] = y00;
                 sm.A[pa * kLd + qb] = y01;
                 sm.A[qa * kLd + pb] = y10;
                 sm.A[qa * kLd + qb] = y11;
                 // V <- V J_b on rows 2*pa_idx, 2*pa_idx + 1
-#pragma unroll
-                for (int rr = 0; rr < 2; ++rr) {
-                    const int row = 2 * pa_idx + rr;
-                    const double v0 = sm.V[row * kLd + pb], v1 = sm.V[row * kLd + qb];
-                    sm.V[row * kLd + pb] = cb * v0 - sb * v1;
-                    sm.V[row * kLd + qb] = sb * v0 + cb * v1;
-                }
+                sm.V[(2 * pa_idx) * kLd + pb] = cb * v00 - sb * v01;
+                sm.V[(2 * pa_idx) * kLd + qb] = sb * v00 + cb * v01;
+                sm.V[(2 * pa_idx + 1) * kLd + pb] = cb * v10 - sb * v11;
+                sm.V[(2 * pa_idx + 1) * kLd + qb] = sb * v10 + cb * v11;
             }
-            __syncthreads();
+            asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
+            // next round: every index except the fixed one (N) moves one step
+            if (a0 != N && ++a0 == N) a0 = 0;
+            if (++a1 == N) a1 = 0;
+            if (b0 != N && ++b0 == N) b0 = 0;
+            if (++b1 == N) b1 = 0;
         }
         ++sweeps;
+        // converged when no off-diagonal element exceeds the threshold (one pass over the matrix)
+        int big = 0;
+        for (int e = tid; e < M2 * M2; e += jthreads) {
+            const int k = e / M2, l = e % M2;
+            big |= (k != l) && (fabs(sm.A[k * kLd + l]) > thresh);
+        }
+        big = __any_sync(0xffffffffu, big);
+        if (big && (tid & 31) == 0) sm.flag_rotated = 1;
+        asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
         const int rotated = sm.flag_rotated;
-        __syncthreads();  // everyone has read the flag
+        asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");  // everyone has read the flag
         if (!rotated) converged = true;
         if (tid == 0) sm.flag_rotated = 0;
-        __syncthreads();  // reset is visible before the next sweep can set it again
+        // the barriers of the next sweep's first round order this reset before the next set
     }
 
     // ---------------------------------------------------------------- phase 4: sigma, j, d, c
@@ -268,7 +298,7 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
         const double mu = sm.A[tid * kLd + tid];
         sm.mu[tid] = mu > QN_NOISE_FLOOR * sm.diag_scale ? mu : 0.0;
     }
-    __syncthreads();
+    asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
     if (tid < m) {
         const double mine = sm.mu[tid];
         int rank = 0;
@@ -279,7 +309,7 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
         sm.order[rank] = tid;
         sm.sigma[rank] = sqrt(mine > 0.0 ? mine : 0.0);
     }
-    __syncthreads();
+    asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
     if (tid == 0) {
         int j = 0;
         const double s1 = sm.sigma[0];
@@ -288,7 +318,7 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
         if (j > m - 1) j = m - 1;
         sm.j = j;
     }
-    __syncthreads();
+    asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
     const int j = sm.j;
     if (tid < j) {
         const int col = sm.order[tid];
@@ -296,13 +326,13 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
         for (int k = 0; k < m; ++k) dot += sm.V[k * kLd + col] * sm.w[k];
         sm.modec[tid] = dot / sm.mu[col];
     }
-    __syncthreads();
+    asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
     if (tid < m) {
         double dk = 0.0;
         for (int r = 0; r < j; ++r) dk += sm.V[tid * kLd + sm.order[r]] * sm.modec[r];
         sm.d[tid] = dk;
     }
-    __syncthreads();
+    asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
     if (tid < QN_MAX_M) {
         double s = 0.0;
         for (int k = 0; k < m; ++k) s += sm.d[k];
@@ -329,8 +359,8 @@ cudaError_t qn_solve_init() {
 cudaError_t qn_launch_solve(const qn_solve_params& p, cudaStream_t st, int* launches) {
     const int M2 = p.m + (p.m & 1);
     const int H = M2 / 2;
-    int threads = 256;
-    while (threads < H * H) threads <<= 1;
+    (void)H;
+    const int threads = 1024;  // the partial sums and the centring use all of them; the Jacobi phase H*H
     qn::solve_kernel<<<1, threads, sizeof(qn::SolveSmem), st>>>(p);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess && launches) *launches += 1;
