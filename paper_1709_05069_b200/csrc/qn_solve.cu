@@ -172,10 +172,8 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
 
     // ---------------------------------------------------------------- phase 3: two-sided Jacobi
     // Round-robin ordering: M2/2 disjoint pairs per round, M2-1 rounds per sweep.  Thread (a, b) owns
-    // the 2x2 block (rows of pair a) x (columns of pair b) for the round.  It reads the diagonal blocks
-    // of its two pairs and its own block, everybody synchronises, and it then computes BOTH rotations
-    // itself (the same numbers in every thread that needs them) and writes its block: two barriers per
-    // round and no separate "compute the angles" phase on the critical path.
+    // the 2x2 block (rows of pair a) x (columns of pair b) for the round; the threads on the diagonal
+    // (a == b) first compute their pair's rotation and publish (c, s).  Two barriers per round.
     const int M2 = m + (m & 1);
     const int H = M2 / 2;
     const int N = M2 - 1;
@@ -204,56 +202,49 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
     int b0 = pb_idx == 0 ? N : pb_idx % N, b1 = pb_idx == 0 ? 0 : (N - pb_idx) % N;
     int sweeps = 0;
     bool converged = (fro == 0.0) || m < 2;
+    // Rotation that zeroes a_pq.  The angle comes from fp32 arithmetic on values scaled into fp32 range
+    // (two MUFU reciprocal-square-roots and one reciprocal; relative error ~1e-7), so the rotation leaves
+    // a'_pq = O(1e-7 a_pq), which the next sweep removes.  What must hold to fp64 accuracy is
+    // c^2 + s^2 = 1: (c, s) are rescaled in fp64 by 1 - e/2 with e = c^2 + s^2 - 1 ~ 1e-7, which leaves
+    // an error of 3e^2/8 ~ 4e-15 per rotation.  fp64 operations have a long dependent latency on this
+    // part, so as few as possible sit on this chain.
     auto rotation = [&](double app, double aqq, double apq, double& c, double& s) {
         c = 1.0;
         s = 0.0;
         if (fabs(apq) > thresh) {
-            // tan of the rotation angle from fp32 arithmetic (relative error ~1e-7): the rotation then
-            // leaves a'_pq = O(1e-7 a_pq) instead of 0, which the next sweep removes.  What must hold to
-            // fp64 accuracy is c^2 + s^2 = 1: c = rsqrt(1 + t^2) is refined by two Newton steps.
-            const float zeta = (float)((aqq - app) * inv_fro) / (2.0f * (float)(apq * inv_fro));
-            const float tf = copysignf(1.0f, zeta) / (fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.0f)));
-            const double t = (double)tf;
-            const double x = fma(t, t, 1.0);
-            double y = (double)rsqrtf((float)x);
-            y = y * fma(-0.5 * x, y * y, 1.5);
-            y = y * fma(-0.5 * x, y * y, 1.5);
-            c = y;
-            s = t * y;
+            const float df = (float)((aqq - app) * inv_fro);
+            const float of = (float)((apq + apq) * inv_fro);
+            const float r2 = fmaf(df, df, of * of);
+            const float h = r2 * rsqrtf(r2);                                   // sqrt(d^2 + o^2)
+            const float tf = copysignf(__fdividef(fabsf(of), fabsf(df) + h), df * of);  // tan(phi)
+            const float cf = rsqrtf(fmaf(tf, tf, 1.0f));
+            const double c0 = (double)cf, s0 = (double)(tf * cf);
+            const double e = fma(c0, c0, fma(s0, s0, -1.0));
+            const double k = fma(e, -0.5, 1.0);
+            c = c0 * k;
+            s = s0 * k;
         }
     };
     while (!converged && sweeps < kMaxSweeps) {
         for (int r = 0; r < N; ++r) {
-            double ca = 1.0, sa = 0.0, cb = 1.0, sb = 0.0;
-            double x00 = 0, x01 = 0, x10 = 0, x11 = 0, v00 = 0, v01 = 0, v10 = 0, v11 = 0;
-            double daa_pp = 0, daa_qq = 0, daa_pq = 0, dbb_pp = 0, dbb_qq = 0, dbb_pq = 0;
             const int pa = a0 < a1 ? a0 : a1, qa = a0 < a1 ? a1 : a0;
             const int pb = b0 < b1 ? b0 : b1, qb = b0 < b1 ? b1 : b0;
-            if (worker) {
-                daa_pp = sm.A[pa * kLd + pa];
-                daa_qq = sm.A[qa * kLd + qa];
-                daa_pq = sm.A[pa * kLd + qa];
-                dbb_pp = sm.A[pb * kLd + pb];
-                dbb_qq = sm.A[qb * kLd + qb];
-                dbb_pq = sm.A[pb * kLd + qb];
-                x00 = sm.A[pa * kLd + pb];
-                x01 = sm.A[pa * kLd + qb];
-                x10 = sm.A[qa * kLd + pb];
-                x11 = sm.A[qa * kLd + qb];
-                v00 = sm.V[(2 * pa_idx) * kLd + pb];
-                v01 = sm.V[(2 * pa_idx) * kLd + qb];
-                v10 = sm.V[(2 * pa_idx + 1) * kLd + pb];
-                v11 = sm.V[(2 * pa_idx + 1) * kLd + qb];
+            // the thread on the diagonal block of pair a computes that pair's rotation for everybody
+            if (worker && pa_idx == pb_idx) {
+                double c, s2;
+                rotation(sm.A[pa * kLd + pa], sm.A[qa * kLd + qa], sm.A[pa * kLd + qa], c, s2);
+                sm.rot_c[pa_idx] = c;
+                sm.rot_s[pa_idx] = s2;
             }
-            asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");  // all reads done before any write
+            asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
             if (worker) {
-                rotation(daa_pp, daa_qq, daa_pq, ca, sa);
-                if (pa_idx == pb_idx) {
-                    cb = ca;
-                    sb = sa;
-                } else {
-                    rotation(dbb_pp, dbb_qq, dbb_pq, cb, sb);
-                }
+                const double ca = sm.rot_c[pa_idx], sa = sm.rot_s[pa_idx];
+                const double cb = sm.rot_c[pb_idx], sb = sm.rot_s[pb_idx];
+                const double x00 = sm.A[pa * kLd + pb], x01 = sm.A[pa * kLd + qb];
+                const double x10 = sm.A[qa * kLd + pb], x11 = sm.A[qa * kLd + qb];
+                const double v00 = sm.V[(2 * pa_idx) * kLd + pb], v01 = sm.V[(2 * pa_idx) * kLd + qb];
+                const double v10 = sm.V[(2 * pa_idx + 1) * kLd + pb], v11 = sm.V[(2 * pa_idx + 1) * kLd + qb];
+                // Y = J_a^T X J_b on this thread's 2x2 block (only this thread touches these four entries)
                 const double t00 = cb * x00 - sb * x01, t01 = sb * x00 + cb * x01;
                 const double t10 = cb * x10 - sb * x11, t11 = sb * x10 + cb * x11;
                 double y00 = ca * t00 - sa * t10, y10 = sa * t00 + ca * t10;
