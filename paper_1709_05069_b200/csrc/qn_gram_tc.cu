@@ -24,11 +24,11 @@
 // t is accumulated by the CUDA cores that build the tiles (fp32 products, fp64 every tile).
 //
 // Structure (one persistent CTA per SM, warp-specialised):
-//   warps 0-3   drain warps: tcgen05.ld their TMEM quadrant (one D row per thread), fold the hi and lo
+//   warps 4-7   drain warps: tcgen05.ld their TMEM quadrant (one D row per thread), fold the hi and lo
 //               column halves and add into per-thread fp32 accumulators; fp64 in shared memory every 16
 //               drains; the two row halves are added at the end
-//   warp  4     one lane issues tcgen05.mma / tcgen05.commit
-//   warps 5..   producer warps: 128-bit global loads -> registers -> mean by shuffles -> hi/lo split
+//   warp  3     one lane issues tcgen05.mma / tcgen05.commit
+//   others      producer warps: 128-bit global loads -> registers -> mean by shuffles -> hi/lo split
 //               -> swizzled st.shared; one K tile (64 columns) per warp at a time, stages double-buffered
 // Stages and accumulator buffers are handed over with mbarriers.  Every wait has an iteration limit:
 // when it runs out the CTA sets an abort flag and an error word, stops waiting, finishes its loops,
@@ -95,11 +95,15 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false (and raises the abort flag) when the limit runs out or another thread
 // of the CTA has already given up.
+template <bool kBackOff = true>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
     if (mbar_try(bar, parity)) return true;  // the common case costs one shared-memory round trip
     if (*abort) return false;
     for (uint32_t it = 0; it < kTcWaitLimit; ++it) {
         if (mbar_try(bar, parity)) return true;
+        // waiting producer and drain warps sleep between polls so that they do not take issue slots from
+        // the MMA warp; the MMA warp itself polls without sleeping
+        if (kBackOff) __nanosleep(64);
         if ((it & 255u) == 255u && *abort) return false;
     }
     *abort = 1;
@@ -155,6 +159,10 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     volatile int* abort = &sm.abort;
+    // Roles by warp: 3 = MMA issue (alone with one drain and one producer warp on its scheduler), 4..7 = drain
+    // (TMEM quadrant = warp - 4 = warp % 4), the rest = producers.
+    constexpr int kMmaWarp = 3, kDrainWarp0 = 4;
+    const bool is_drain = warp >= kDrainWarp0 && warp < kDrainWarp0 + 4;
 
     // Tiles of 64 columns are dealt round-robin to the CTAs; a CTA's tiles are grouped U per stage, and
     // the count is padded to a multiple of U with all-zero tiles (they add nothing).
@@ -176,7 +184,7 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
         sm.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 4) {
+    if (warp == kMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
                      "r"(kTmemCols)
                      : "memory");
@@ -187,11 +195,13 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = sm.tmem_base;
 
-    if (warp < 4) {
+    if (is_drain) {
         // ------------------------------------------------------------------ drain warps
+        const int dq = warp - kDrainWarp0;  // TMEM quadrant of this warp
+        const int dtid = dq * 32 + lane;
         // D is 128 x 128 (M = 128: row i in TMEM lane i).  Row r belongs to tile r / RT of the stage and
         // needs that tile's own RT columns only: D[r][cb + c] (hi columns) + D[r][cb + MP + c] (lo columns).
-        const int row = tid;
+        const int row = dtid;
         const uint32_t cb = (uint32_t)((row / RT) * RT);
         float facc[MP];
 #pragma unroll
@@ -209,7 +219,7 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
 #pragma unroll
             for (int c0 = 0; c0 < MP; c0 += 32) {
                 uint32_t v0[16], v1[16], u0[16], u1[16];
-                const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(b * 128) + cb + c0;
+                const uint32_t taddr = tmem_base + ((uint32_t)(dq * 32) << 16) + (uint32_t)(b * 128) + cb + c0;
                 TC_LD16(v0, taddr);
                 TC_LD16(v1, taddr + 16);
                 TC_LD16(u0, taddr + MP);
@@ -238,7 +248,7 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
                 }
             }
         }
-    } else if (warp == 4) {
+    } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issue
         if (lane == 0) {
             // kind::f16, fp32 accumulate, bf16 x bf16, both K-major, N = 128, M = 128
@@ -252,10 +262,10 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
             for (int p = 0; p < nstages; ++p) {
                 const bool first = in_chain == 0;
                 if (first) {
-                    mbar_wait(&sm.accempty[b], acc_par ^ 1u, abort);
+                    mbar_wait<false>(&sm.accempty[b], acc_par ^ 1u, abort);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 }
-                mbar_wait(&sm.full[s], full_par, abort);
+                mbar_wait<false>(&sm.full[s], full_par, abort);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 // the start-address field counts 16-byte units: a stage is 16 KB, a K step of 16 bf16 is 32 B
                 const uint64_t desc = desc0 + (uint64_t)(s * (16384 >> 4));
@@ -294,7 +304,7 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
         // Work item = RPT rows x 8 columns per thread (8 sixteen-byte loads): the warp's lanes are CH
         // column chunks x RQ row groups, a tile takes PASSES items.  The loads of the next item are
         // issued before the current one is processed, so a warp always has loads in flight.
-        const int pw = warp - 5;
+        const int pw = warp < kMmaWarp ? warp : warp - 5;
         const int rq = lane / CH, cl = lane % CH;
         const int row0 = rq * RPT;
         // bf16, MP = 64: two row groups share a quarter-warp; the odd one walks its rows in the order
@@ -433,7 +443,7 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
         out[m * (m + 1) / 2 + tid] = poisoned ? qnan : s;
     }
     if (tid == 0 && *abort && error_word) atomicExch(error_word, 1);
-    if (warp == 4) {
+    if (warp == kMmaWarp) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
