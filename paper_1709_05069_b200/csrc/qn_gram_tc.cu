@@ -45,7 +45,7 @@ template <int MP>
 struct TcShape {
     static constexpr int kTilesPerStage = MP == 32 ? 2 : 1;
     static constexpr int kProducers = MP == 32 ? 10 : 7;
-    static constexpr int kStages = MP == 32 ? 10 : 9;
+    static constexpr int kStages = MP == 32 ? 10 : 8;
     static constexpr int kThreads = (4 + 1 + kProducers) * 32;
 };
 
@@ -69,8 +69,7 @@ struct TcSmem {
     double acc64[MP * 128];  // [Gram column][D row], fp64 sums of the folded rows
     double tpart[kProducers][MP];
     alignas(8) uint64_t full[kStages];
-    uint64_t empty[kStages];
-    uint64_t accfull[4];
+    uint64_t done[kStages];  // one per group of stages (only the first kStages / group size are used)
     uint64_t accempty[4];
     uint32_t tmem_base;
     int abort;
@@ -145,7 +144,9 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
     constexpr int U = TcShape<MP>::kTilesPerStage;           // tiles sharing a 128-row stage
     constexpr int kStages = TcShape<MP>::kStages;
     constexpr int kProducers = TcShape<MP>::kProducers;
-    constexpr int kDrainEvery = TcFlush<T, MP>::kStagesPerDrain;
+    constexpr int kDrainEvery = TcFlush<T, MP>::kStagesPerDrain;  // stages per group = per accumulation chain
+    constexpr int kGroups = kStages / kDrainEvery;                // groups in the shared-memory ring
+    static_assert(kStages % kDrainEvery == 0, "the ring holds whole groups");
     constexpr int LD = sizeof(T) == 2 ? 1 : 2;  // 16-byte loads per 8-column chunk of one row
     constexpr int RPT = 8 / LD;        // rows per producer thread: 8 loads per work item either way
     constexpr int RQ = MP / RPT;       // row groups across the lanes of a producer warp
@@ -175,10 +176,9 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&sm.full[s], U);
-            mbar_init(&sm.empty[s], 1);
+            mbar_init(&sm.done[s], 1);
         }
         for (int b = 0; b < kAccBufs; ++b) {
-            mbar_init(&sm.accfull[b], 1);
             mbar_init(&sm.accempty[b], 4);
         }
         sm.abort = 0;
@@ -209,10 +209,10 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
 #pragma unroll 4
         for (int e = 0; e < MP; ++e) sm.acc64[e * 128 + row] = 0.0;
         const int ndrains = (int)ndrain;
-        int b = 0, since_wide = 0;
-        uint32_t acc_par = 0;
+        int b = 0, since_wide = 0, gs = 0;
+        uint32_t done_par = 0;
         for (int f = 0; f < ndrains; ++f) {
-            mbar_wait(&sm.accfull[b], acc_par, abort);
+            mbar_wait(&sm.done[gs], done_par, abort);  // the group's MMAs have completed
             __syncwarp();
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             // 32 Gram columns per round: hi and lo halves, four 16-column loads in flight, one wait
@@ -235,9 +235,10 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.accempty[b]);
-            if (++b == kAccBufs) {
-                b = 0;
-                acc_par ^= 1u;
+            if (++b == kAccBufs) b = 0;
+            if (++gs == kGroups) {
+                gs = 0;
+                done_par ^= 1u;
             }
             if (++since_wide == kTcWideEvery || f == ndrains - 1) {
                 since_wide = 0;
@@ -257,7 +258,7 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
             // CTA, so stage index, parities and descriptors are carried along instead of recomputed.
             const uint64_t desc0 = tc_smem_desc(smem_u32(sm.stage[0]));
             const int nstages = (int)my_stages;
-            int s = 0, b = 0, in_chain = 0;
+            int s = 0, b = 0, in_chain = 0, gs = 0;
             uint32_t full_par = 0, acc_par = 0;
             for (int p = 0; p < nstages; ++p) {
                 const bool first = in_chain == 0;
@@ -279,14 +280,15 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
                         "l"(desc + 2 * k), "l"(desc + 2 * k), "r"(idesc), "r"(accumulate)
                         : "memory");
                 }
-                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
-                                 smem_u32(&sm.empty[s]))
-                             : "memory");
+                // One commit per group: a commit stalls the tensor pipe for about 430 cycles, so the same
+                // mbarrier tells the producers that the group's stages are free and the drain warps that
+                // the group's accumulator is complete.
                 if (++in_chain == kDrainEvery || p == nstages - 1) {
                     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
-                                     smem_u32(&sm.accfull[b]))
+                                     smem_u32(&sm.done[gs]))
                                  : "memory");
                     in_chain = 0;
+                    if (++gs == kGroups) gs = 0;
                     if (++b == kAccBufs) {
                         b = 0;
                         acc_par ^= 1u;
@@ -370,7 +372,7 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
 #pragma unroll
                 for (int e = 0; e < 8; ++e) r[e] *= inv_m;
                 if (pass == 0)  // the stage must have been consumed by the MMAs of its previous use
-                    mbar_wait(&sm.empty[s], (uint32_t)(((p / kStages) & 1) ^ 1), abort);
+                    mbar_wait(&sm.done[(p / kDrainEvery) % kGroups], (uint32_t)(((p / kStages) & 1) ^ 1), abort);
 #pragma unroll
                 for (int j = 0; j < RPT; ++j) {
                     const int row = row0 + (j ^ sw);
