@@ -5,8 +5,11 @@
 // update after each Write but does not say what the Server keeps; the window and its raw Gram are
 // this library's reading.)
 //
-// The raw Gram has to carry the cancellation of the later m x m centring, so every product is
-// formed and accumulated in fp64 (products of two fp32 or bf16 values are exact in fp64).
+// The raw Gram has to carry the cancellation of the later m x m centring.  Two arithmetic modes, as in
+// the Gram pass: kPrecise (n < QN_PRECISE_BELOW) forms and adds every product in fp64 (a product of two
+// fp32 or bf16 values is exact in fp64); the fast mode adds the products of one work item (4 or 8 columns)
+// in fp32 starting from zero and then goes to fp64 -- eight times fewer fp32->fp64 conversions, which is
+// what bounds the precise mode; its rounding errors are unbiased and average out as 1/sqrt(n).
 // The last CTA to finish adds the per-CTA partial rows in a fixed order and patches row and column
 // `slot` of the Gram: no CTA ever waits for another.
 #include "qn_device.cuh"
@@ -16,7 +19,7 @@ namespace qn {
 constexpr int kRowThreads = 256;
 constexpr int kRowBlock = 8;  // window columns handled by one CTA row (blockIdx.y)
 
-template <typename T, bool kAligned>
+template <typename T, bool kAligned, bool kPrecise>
 __global__ void __launch_bounds__(kRowThreads)
 row_kernel(const T* __restrict__ window_g, const T* __restrict__ g_col, T* __restrict__ window_row_out, int64_t n,
            int m, int slot, double* __restrict__ partials, double* __restrict__ raw_gram, unsigned int* ticket) {
@@ -55,14 +58,29 @@ row_kernel(const T* __restrict__ window_g, const T* __restrict__ g_col, T* __res
             else
                 window_row_out[i0] = g_col[i0];
         }
+        if (kPrecise) {
 #pragma unroll
-        for (int e = 0; e < kCols; ++e) {
-            const double a = (double)(kAligned ? Storage<T>::get(xn, e) : __uint_as_float(xn.x));
+            for (int e = 0; e < kCols; ++e) {
+                const double a = (double)(kAligned ? Storage<T>::get(xn, e) : __uint_as_float(xn.x));
 #pragma unroll
-            for (int r = 0; r < kRowBlock; ++r) {
-                const double b = (double)(kAligned ? Storage<T>::get(xl[r], e) : __uint_as_float(xl[r].x));
-                acc[r] = fma(a, b, acc[r]);
+                for (int r = 0; r < kRowBlock; ++r) {
+                    const double b = (double)(kAligned ? Storage<T>::get(xl[r], e) : __uint_as_float(xl[r].x));
+                    acc[r] = fma(a, b, acc[r]);
+                }
             }
+        } else {
+            float part[kRowBlock];
+#pragma unroll
+            for (int r = 0; r < kRowBlock; ++r) part[r] = 0.f;
+#pragma unroll
+            for (int e = 0; e < kCols; ++e) {
+                const float a = kAligned ? Storage<T>::get(xn, e) : __uint_as_float(xn.x);
+#pragma unroll
+                for (int r = 0; r < kRowBlock; ++r)
+                    part[r] = fmaf(a, kAligned ? Storage<T>::get(xl[r], e) : __uint_as_float(xl[r].x), part[r]);
+            }
+#pragma unroll
+            for (int r = 0; r < kRowBlock; ++r) acc[r] += (double)part[r];
         }
     }
 
@@ -122,12 +140,16 @@ static cudaError_t launch_row_t(const T* window_g, const T* g_col, T* window_row
     if (cap > max_partials) cap = max_partials;
     const int gx = (int)(want < cap ? (want > 0 ? want : 1) : cap);
     dim3 grid(gx, nby);
-    if (aligned)
-        row_kernel<T, true><<<grid, kRowThreads, 0, st>>>(window_g, g_col, window_row_out, n, m, slot, partials,
-                                                         raw_gram, ticket);
+    const bool precise = n < QN_PRECISE_BELOW;
+    if (aligned && !precise)
+        row_kernel<T, true, false><<<grid, kRowThreads, 0, st>>>(window_g, g_col, window_row_out, n, m, slot, partials,
+                                                                raw_gram, ticket);
+    else if (aligned)
+        row_kernel<T, true, true><<<grid, kRowThreads, 0, st>>>(window_g, g_col, window_row_out, n, m, slot, partials,
+                                                               raw_gram, ticket);
     else
-        row_kernel<T, false><<<grid, kRowThreads, 0, st>>>(window_g, g_col, window_row_out, n, m, slot, partials,
-                                                          raw_gram, ticket);
+        row_kernel<T, false, true><<<grid, kRowThreads, 0, st>>>(window_g, g_col, window_row_out, n, m, slot, partials,
+                                                                raw_gram, ticket);
     return cudaGetLastError();
 }
 
