@@ -209,7 +209,12 @@ static cudaError_t launch_combine_t(const T* theta, const T* g, int64_t n, int m
                          (reinterpret_cast<uintptr_t>(out) % 16 == 0) && ((n * (int64_t)sizeof(T)) % 16 == 0);
     const int64_t nitems = aligned ? n / Storage<T>::kVec : n;
     const int64_t want = (nitems + kCombineThreads - 1) / kCombineThreads;
-    const int64_t cap = (int64_t)qn_sm_count() * 8;
+    int per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, combine_vec_kernel<T>, kCombineThreads, 0) != cudaSuccess ||
+        per_sm < 1)
+        per_sm = 1;
+    // whole waves only: a grid-strided loop gains nothing from a partial last wave
+    const int64_t cap = (int64_t)qn_sm_count() * per_sm * 2;
     const int grid = (int)(want < cap ? (want > 0 ? want : 1) : cap);
     if (aligned)
         combine_vec_kernel<T><<<grid, kCombineThreads, 0, st>>>(theta, g, n, m, coef, out);

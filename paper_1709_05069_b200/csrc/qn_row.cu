@@ -134,8 +134,19 @@ static cudaError_t launch_row_t(const T* window_g, const T* g_col, T* window_row
                          (reinterpret_cast<uintptr_t>(g_col) % 16 == 0) && ((n * (int64_t)sizeof(T)) % 16 == 0);
     const int64_t nitems = aligned ? n / Storage<T>::kVec : n;
     const int nby = (m + kRowBlock - 1) / kRowBlock;
+    // one wave of CTAs: every resident slot of every SM gets one CTA (the loop is grid-strided, so a second,
+    // partial wave would run at a fraction of the occupancy for as long as the first)
+    int per_sm = 1;
+    {
+        const bool precise_q = n < QN_PRECISE_BELOW;
+        cudaError_t oe = aligned && !precise_q
+                             ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_kernel<T, true, false>, kRowThreads, 0)
+                             : aligned ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_kernel<T, true, true>, kRowThreads, 0)
+                                       : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_kernel<T, false, true>, kRowThreads, 0);
+        if (oe != cudaSuccess || per_sm < 1) per_sm = 1;
+    }
     int64_t want = (nitems + kRowThreads - 1) / kRowThreads;
-    int64_t cap = (int64_t)qn_sm_count() * 4 / nby;
+    int64_t cap = (int64_t)qn_sm_count() * per_sm / nby;
     if (cap < 1) cap = 1;
     if (cap > max_partials) cap = max_partials;
     const int gx = (int)(want < cap ? (want > 0 ? want : 1) : cap);
