@@ -119,6 +119,20 @@ class ClockSampler(threading.Thread):
         }
 
 
+def max_over_ranks(x: float, world: int, device) -> float:
+    """The slowest rank's figure: ranks are independent replicas, the job is as slow as its slowest one."""
+    if world <= 1:
+        return float(x)
+    t = torch.tensor([x], device=device, dtype=torch.float64)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(ms_per_step: float, world: int) -> float:
+    """updates/s of the whole job: every rank finishes one update per step (weak scaling, replicas only)."""
+    return world * 1e3 / ms_per_step
+
+
 def dist_env():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -281,12 +295,9 @@ def main():
     timing = qn.qn_timing_end(h)
     launches = h.total_launches - launches0
     status = qn.qn_status_sync(h)
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, dev)
     ms_per_step = total_ms / args.steps
-    value = world * 1e3 / ms_per_step
+    value = whole_job_value(ms_per_step, world)
 
     # dominant kernel and its roofline
     per_kernel = {k: (ms / cnt if cnt else 0.0, cnt) for k, (ms, cnt) in timing.items()}
@@ -319,10 +330,7 @@ def main():
                 qn.qn_update_host(h, th_h, g_h, cfg.tau, cfg.lam, out_h)
             torch.cuda.synchronize()
             dt = (time.perf_counter() - t0) / args.e2e_steps
-            if world > 1:
-                t = torch.tensor([dt], device=dev, dtype=torch.float64)
-                torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-                dt = float(t.item())
+            dt = max_over_ranks(dt, world, dev)
             e2e = {"value": world / dt, "unit": UNIT, "h2d_bytes_per_step": 2 * cfg.m * cfg.n * cfg.elem_bytes,
                    "d2h_bytes_per_step": cfg.n * cfg.elem_bytes + 528, "ms_per_step": dt * 1e3,
                    "steps": args.e2e_steps, "api": "qn_update_host (pinned host buffers in, theta_new + j + sigma out)"}
