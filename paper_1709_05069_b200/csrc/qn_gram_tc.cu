@@ -44,7 +44,7 @@ namespace qn {
 template <int MP>
 struct TcShape {
     static constexpr int kTilesPerStage = MP == 32 ? 2 : 1;
-    static constexpr int kProducers = MP == 32 ? 10 : 7;
+    static constexpr int kProducers = MP == 32 ? 11 : 7;
     static constexpr int kStages = MP == 32 ? 10 : 8;
     static constexpr int kThreads = (4 + 1 + kProducers) * 32;
 };
@@ -67,7 +67,6 @@ struct TcSmem {
     static constexpr int kProducers = TcShape<MP>::kProducers;
     alignas(1024) unsigned char stage[kStages][128 * 128];
     double acc64[MP * 128];  // [Gram column][D row], fp64 sums of the folded rows
-    double tpart[kProducers][MP];
     alignas(8) uint64_t full[kStages];
     uint64_t done[kStages];  // one per group of stages (only the first kStages / group size are used)
     uint64_t accempty[4];
@@ -126,6 +125,21 @@ __device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo_elem, float hi_elem)
     return w;
 }
 
+// Packed pairs of fp32 (one 64-bit register, two lanes of the fp32 pipe per instruction).
+__device__ __forceinline__ uint64_t pk2(float lo, float hi) {
+    uint64_t v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+    return v;
+}
+__device__ __forceinline__ void unpk2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
 // 16 consecutive fp32 columns of this thread's TMEM lane into r[0..15]
 #define TC_LD16(r, taddr)                                                                                      \
     asm volatile(                                                                                              \
@@ -147,11 +161,7 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
     constexpr int kDrainEvery = TcFlush<T, MP>::kStagesPerDrain;  // stages per group = per accumulation chain
     constexpr int kGroups = kStages / kDrainEvery;                // groups in the shared-memory ring
     static_assert(kStages % kDrainEvery == 0, "the ring holds whole groups");
-    constexpr int LD = sizeof(T) == 2 ? 1 : 2;  // 16-byte loads per 8-column chunk of one row
-    constexpr int RPT = 8 / LD;        // rows per producer thread: 8 loads per work item either way
-    constexpr int RQ = MP / RPT;       // row groups across the lanes of a producer warp
-    constexpr int CH = 32 / RQ;        // 8-column chunks handled side by side
-    constexpr int PASSES = 8 / CH;     // work items per thread per tile
+    constexpr int LD = sizeof(T) == 2 ? 1 : 2;  // 16-byte registers per 8-column chunk of one row
     constexpr uint32_t kTmemCols = 512;  // four accumulator buffers of 128 fp32 columns: all of TMEM
     constexpr int kAccBufs = 4;
     static_assert(U * RT == 128, "a stage is 128 operand rows");
@@ -190,6 +200,10 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    // operand rows >= m (hi and lo) are never written by the producers and must read as zero
+    for (int o = tid * 16; o < kStages * 128 * 128; o += TcShape<MP>::kThreads * 16)
+        *reinterpret_cast<uint4*>(&sm.stage[0][0] + o) = make_uint4(0, 0, 0, 0);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -303,118 +317,82 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ producer warps
-        // Work item = RPT rows x 8 columns per thread (8 sixteen-byte loads): the warp's lanes are CH
-        // column chunks x RQ row groups, a tile takes PASSES items.  The loads of the next item are
-        // issued before the current one is processed, so a warp always has loads in flight.
+        // The warp's lanes are 8 column chunks (8 columns each: one whole 64-column row segment per
+        // load instruction) x 4 row groups; a thread handles 8 rows of one chunk per item and a tile
+        // takes MP / 32 items.  Rows are independent of one another (the reference is Worker 0's row,
+        // read once per item), so an item's registers are reloaded row by row, each as soon as its row
+        // has been converted and stored: a warp keeps loads in flight through the conversion without a
+        // second set of registers.  Rows >= m are never written; the stages are zeroed once at the start.
         const int pw = warp < kMmaWarp ? warp : warp - 5;
-        const int rq = lane / CH, cl = lane % CH;
-        const int row0 = rq * RPT;
-        // bf16, MP = 64: two row groups share a quarter-warp; the odd one walks its rows in the order
-        // 4,5,6,7,0,1,2,3 so that the two groups' 16-byte stores land on different swizzle positions.
-        const int sw = (RPT == 8 && CH == 4) ? ((rq & 1) << 2) : 0;
-        const float inv_m = 1.0f / (float)m;
-        float tacc[RPT];
-        double tacc64[RPT];
+        const int rq = lane >> 3, cl = lane & 7;
+        uint4 raw[8][LD], ref[LD], ref_next[LD];
+        auto load_chunk = [&](uint4 (&dst)[LD], int row, int64_t q) {
+            const int64_t i0 = (blockIdx.x + q * (int64_t)gridDim.x) * kTcTileCols + cl * 8;
 #pragma unroll
-        for (int j = 0; j < RPT; ++j) {
-            tacc[j] = 0.f;
-            tacc64[j] = 0.0;
-        }
-        auto issue_loads = [&](uint4 (&raw)[RPT][LD], int64_t q, int pass) {
-            const int64_t i0 = (blockIdx.x + q * (int64_t)gridDim.x) * kTcTileCols + (cl + CH * pass) * 8;
-#pragma unroll
-            for (int j = 0; j < RPT; ++j) {
-                const int row = row0 + (j ^ sw);
-#pragma unroll
-                for (int l = 0; l < LD; ++l) raw[j][l] = make_uint4(0, 0, 0, 0);
-                if (q < my_tiles && row < m && i0 < n) {
-                    // rows are 32-byte aligned and n is a multiple of 8 on this path (see
-                    // qn_gram_tc_applicable), so an 8-column chunk is never cut by the end of the row
-                    if (LD == 1)
-                        raw[j][0] = ldg_stream16(g + (int64_t)row * n + i0);
-                    else
-                        ldg_stream32(g + (int64_t)row * n + i0, raw[j][0], raw[j][LD - 1]);
-                }
+            for (int l = 0; l < LD; ++l) dst[l] = make_uint4(0, 0, 0, 0);
+            if (q < my_tiles && i0 < n) {
+                // rows are 32-byte aligned and n is a multiple of 8 on this path (see
+                // qn_gram_tc_applicable), so an 8-column chunk is never cut by the end of the row
+                if (LD == 1)
+                    dst[0] = ldg_stream16(g + (int64_t)row * n + i0);
+                else
+                    ldg_stream32(g + (int64_t)row * n + i0, dst[0], dst[LD - 1]);
             }
         };
-        uint4 nxt[RPT][LD];
-        issue_loads(nxt, pw, 0);
+        load_chunk(ref, 0, pw);
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (rq * 8 + j < m) load_chunk(raw[j], rq * 8 + j, pw);
         for (int64_t q = pw; q < my_tiles_padded; q += kProducers) {
             const int64_t p = q / U;                 // stage use this tile belongs to
             const int s = (int)(p % kStages);
             unsigned char* tile = sm.stage[s] + (int)(q % U) * (RT * 128);
+            load_chunk(ref_next, 0, q + kProducers);
+            // the stage must have been consumed by the MMAs of its previous use
+            mbar_wait(&sm.done[(p / kDrainEvery) % kGroups], (uint32_t)(((p / kStages) & 1) ^ 1), abort);
 #pragma unroll
-            for (int pass = 0; pass < PASSES; ++pass) {
-                const int c = cl + CH * pass;
-                uint4 raw[RPT][LD];
+            for (int rp = 0; rp < MP / 32; ++rp) {
 #pragma unroll
-                for (int j = 0; j < RPT; ++j)
+                for (int j = 0; j < 8; ++j) {
+                    const int row = rp * 32 + rq * 8 + j;
+                    if (row < m) {
+                        uint32_t hw[4], lw[4];
 #pragma unroll
-                    for (int l = 0; l < LD; ++l) raw[j][l] = nxt[j][l];
-                if (pass + 1 < PASSES)
-                    issue_loads(nxt, q, pass + 1);
-                else
-                    issue_loads(nxt, q + kProducers, 0);
-                // column sums over this thread's rows, then over the RQ row groups of the warp
-                float r[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    float sum = 0.f;
-#pragma unroll
-                    for (int j = 0; j < RPT; ++j) sum += Storage<T>::get(raw[j][e / (8 / LD)], e % (8 / LD));
-                    r[e] = sum;
-                }
-#pragma unroll
-                for (int o = CH; o < 32; o <<= 1) {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) r[e] += __shfl_xor_sync(0xffffffffu, r[e], o);
-                }
-#pragma unroll
-                for (int e = 0; e < 8; ++e) r[e] *= inv_m;
-                if (pass == 0)  // the stage must have been consumed by the MMAs of its previous use
-                    mbar_wait(&sm.done[(p / kDrainEvery) % kGroups], (uint32_t)(((p / kStages) & 1) ^ 1), abort);
-#pragma unroll
-                for (int j = 0; j < RPT; ++j) {
-                    const int row = row0 + (j ^ sw);
-                    const bool real = row < m;
-                    float x[8], lo[8];
-                    uint32_t hw[4], lw[4];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const float v = Storage<T>::get(raw[j][e / (8 / LD)], e % (8 / LD));
-                        x[e] = real ? v - r[e] : 0.f;
-                        tacc[j] = fmaf(x[e], r[e], tacc[j]);
+                        for (int pp = 0; pp < 4; ++pp) {
+                            const float v0 = Storage<T>::get(raw[j][pp / (4 / LD)], (2 * pp) % (8 / LD));
+                            const float v1 = Storage<T>::get(raw[j][pp / (4 / LD)], (2 * pp + 1) % (8 / LD));
+                            float r0 = Storage<T>::get(ref[pp / (4 / LD)], (2 * pp) % (8 / LD));
+                            float r1 = Storage<T>::get(ref[pp / (4 / LD)], (2 * pp + 1) % (8 / LD));
+                            if (rp == 0 && j == 0 && rq == 0) r0 = r1 = 0.f;  // operand row 0 carries the reference itself
+                            float x0, x1, l0, l1;
+                            unpk2(sub2(pk2(v0, v1), pk2(r0, r1)), x0, x1);
+                            hw[pp] = pack_bf16x2_rn(x0, x1);
+                            unpk2(sub2(pk2(x0, x1), pk2(__uint_as_float(hw[pp] << 16), __uint_as_float(hw[pp] & 0xffff0000u))),
+                                  l0, l1);
+                            lw[pp] = pack_bf16x2_rn(l0, l1);
+                        }
+                        // this row's registers are free: fetch the same lane's row of the next item into them
+                        if (rp + 1 < MP / 32) {
+                            if (row + 32 < m) load_chunk(raw[j], row + 32, q);
+                        } else {
+                            load_chunk(raw[j], rq * 8 + j, q + kProducers);
+                        }
+                        // operand row `row` (hi) and MP + row (lo); both have the same row & 7
+                        const uint32_t off = (uint32_t)(row * 128 + ((cl ^ (row & 7)) << 4));
+                        *reinterpret_cast<uint4*>(tile + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                        *reinterpret_cast<uint4*>(tile + MP * 128 + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                    } else if (MP == 64 && rp == 1 && rq * 8 + j < m) {
+                        // no such row in this item, but the lane's row of the next tile's first item exists
+                        load_chunk(raw[j], rq * 8 + j, q + kProducers);
                     }
-#pragma unroll
-                    for (int pp = 0; pp < 4; ++pp) {
-                        hw[pp] = pack_bf16x2_rn(x[2 * pp], x[2 * pp + 1]);
-                        lo[2 * pp] = x[2 * pp] - __uint_as_float(hw[pp] << 16);
-                        lo[2 * pp + 1] = x[2 * pp + 1] - __uint_as_float(hw[pp] & 0xffff0000u);
-                        lw[pp] = pack_bf16x2_rn(lo[2 * pp], lo[2 * pp + 1]);
-                    }
-                    // operand row `row` (hi) and MP + row (lo); both have the same row & 7
-                    const uint32_t off = (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4));
-                    *reinterpret_cast<uint4*>(tile + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-                    *reinterpret_cast<uint4*>(tile + MP * 128 + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
                 }
             }
 #pragma unroll
-            for (int j = 0; j < RPT; ++j) {
-                tacc64[j] += (double)tacc[j];
-                tacc[j] = 0.f;
-            }
+            for (int l = 0; l < LD; ++l) ref[l] = ref_next[l];
             // make the generic-proxy stores visible to the tensor core, then hand the tile over
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.full[s]);
-        }
-        // t of this warp: add the CH lanes that share a row group (fixed butterfly order)
-#pragma unroll
-        for (int j = 0; j < RPT; ++j) {
-            double v = tacc64[j];
-#pragma unroll
-            for (int o = 1; o < CH; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            if (cl == 0) sm.tpart[pw][row0 + (j ^ sw)] = v;
         }
     }
 
@@ -424,9 +402,11 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
     const bool poisoned = *abort != 0;
     double* out = partials + (int64_t)blockIdx.x * qn_partial_len(m);
     if (tid < 128) {
-        // C'[a][bc]: hi rows and lo rows of the folded accumulators, over the U tiles of a stage
+        // F[a][bc]: hi rows and lo rows of the folded accumulators, over the U tiles of a stage.  Operand
+        // row 0 is the reference itself, so F[0][bc] = t[bc] and row 0 of C' (Worker 0 minus itself) is 0.
         constexpr int PER = MP * MP / 128;
         const int a = tid % MP, h = tid / MP;
+        const int tri = m * (m + 1) / 2;
 #pragma unroll 4
         for (int e = 0; e < PER; ++e) {
             const int bc = h * PER + e;
@@ -434,15 +414,15 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
                 double v = 0.0;
 #pragma unroll
                 for (int u = 0; u < U; ++u) v += sm.acc64[bc * 128 + u * RT + a] + sm.acc64[bc * 128 + u * RT + MP + a];
-                out[qn_tri_index(m, a, bc)] = poisoned ? qnan : v;
+                if (poisoned) v = qnan;
+                if (a == 0) {
+                    out[tri + bc] = bc == 0 ? (poisoned ? qnan : 0.0) : v;
+                    out[qn_tri_index(m, 0, bc)] = poisoned ? qnan : 0.0;
+                } else {
+                    out[qn_tri_index(m, a, bc)] = v;
+                }
             }
         }
-    }
-    if (tid < m) {
-        double s = 0.0;
-#pragma unroll
-        for (int w = 0; w < kProducers; ++w) s += sm.tpart[w][tid];
-        out[m * (m + 1) / 2 + tid] = poisoned ? qnan : s;
     }
     if (tid == 0 && *abort && error_word) atomicExch(error_word, 1);
     if (warp == kMmaWarp) {
