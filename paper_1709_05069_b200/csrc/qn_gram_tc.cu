@@ -44,7 +44,7 @@ namespace qn {
 template <int MP>
 struct TcShape {
     static constexpr int kTilesPerStage = MP == 32 ? 2 : 1;
-    static constexpr int kProducers = MP == 32 ? 11 : 7;
+    static constexpr int kProducers = 11;
     static constexpr int kStages = MP == 32 ? 10 : 8;
     static constexpr int kThreads = (4 + 1 + kProducers) * 32;
 };
@@ -55,7 +55,7 @@ struct TcShape {
 // storage, every 2 for fp32 storage, whose inputs carry more bits below the hi/lo split.
 template <typename T, int MP>
 struct TcFlush {
-    static constexpr int kStagesPerDrain = MP == 32 ? 2 : (sizeof(T) == 4 ? 2 : 4);
+    static constexpr int kStagesPerDrain = 2;
 };
 constexpr int kTcTileCols = 64;       // K extent of one tile: 64 bf16 = one 128-byte swizzled row
 constexpr int kTcWideEvery = 16;      // drains between fp32 -> fp64 flushes
@@ -179,13 +179,14 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
     // the count is padded to a multiple of U with all-zero tiles (they add nothing).
     const int64_t ntiles = (n + kTcTileCols - 1) / kTcTileCols;
     const int64_t my_tiles = blockIdx.x < ntiles ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    constexpr int H = MP / 32;  // producer work items (32 Workers x 64 columns) per tile
     const int64_t my_stages = (my_tiles + U - 1) / U;
-    const int64_t my_tiles_padded = my_stages * U;
+    const int64_t my_items_padded = my_stages * 2;  // a stage is two items; a missing one is all zeros
     const int64_t ndrain = (my_stages + kDrainEvery - 1) / kDrainEvery;
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(&sm.full[s], U);
+            mbar_init(&sm.full[s], 2);
             mbar_init(&sm.done[s], 1);
         }
         for (int b = 0; b < kAccBufs; ++b) {
@@ -317,16 +318,19 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ producer warps
-        // The warp's lanes are 8 column chunks (8 columns each: one whole 64-column row segment per
-        // load instruction) x 4 row groups; a thread handles 8 rows of one chunk per item and a tile
-        // takes MP / 32 items.  Rows are independent of one another (the reference is Worker 0's row,
-        // read once per item), so an item's registers are reloaded row by row, each as soon as its row
-        // has been converted and stored: a warp keeps loads in flight through the conversion without a
-        // second set of registers.  Rows >= m are never written; the stages are zeroed once at the start.
+        // Work item = 32 rows x 64 columns: a whole tile for MP = 32, a row half of a tile for MP = 64;
+        // either way a stage takes two items, from two warps.  The warp's lanes are 8 column chunks (8
+        // columns each: one whole 64-column row segment per load instruction) x 4 row groups of 8 rows.
+        // Rows are independent of one another (the reference is Worker 0's row, read once per item), so
+        // an item's registers are reloaded row by row, each as soon as its row has been converted and
+        // stored: a warp keeps loads in flight through the conversion without a second set of registers.
+        // Rows >= m are never written; the stages are zeroed once at the start.
         const int pw = warp < kMmaWarp ? warp : warp - 5;
         const int rq = lane >> 3, cl = lane & 7;
         uint4 raw[8][LD], ref[LD], ref_next[LD];
-        auto load_chunk = [&](uint4 (&dst)[LD], int row, int64_t q) {
+        // 8 columns of Worker `row` in the tile that item k belongs to
+        auto load_chunk = [&](uint4 (&dst)[LD], int row, int64_t k) {
+            const int64_t q = k / H;
             const int64_t i0 = (blockIdx.x + q * (int64_t)gridDim.x) * kTcTileCols + cl * 8;
 #pragma unroll
             for (int l = 0; l < LD; ++l) dst[l] = make_uint4(0, 0, 0, 0);
@@ -339,52 +343,49 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
                     ldg_stream32(g + (int64_t)row * n + i0, dst[0], dst[LD - 1]);
             }
         };
+        // first Worker of item k's rows
+        auto first_row = [&](int64_t k) { return (int)(k % H) * 32 + rq * 8; };
         load_chunk(ref, 0, pw);
 #pragma unroll
         for (int j = 0; j < 8; ++j)
-            if (rq * 8 + j < m) load_chunk(raw[j], rq * 8 + j, pw);
-        for (int64_t q = pw; q < my_tiles_padded; q += kProducers) {
-            const int64_t p = q / U;                 // stage use this tile belongs to
+            if (first_row(pw) + j < m) load_chunk(raw[j], first_row(pw) + j, pw);
+        for (int64_t k = pw; k < my_items_padded; k += kProducers) {
+            const int64_t p = k / 2;                 // stage use this item belongs to
             const int s = (int)(p % kStages);
-            unsigned char* tile = sm.stage[s] + (int)(q % U) * (RT * 128);
-            load_chunk(ref_next, 0, q + kProducers);
+            // operand rows of the item's Worker rows: hi part at hi0 + (row % 32), lo part MP rows further
+            const int hi0 = MP == 32 ? (int)(k & 1) * RT : (int)(k & 1) * 32;
+            unsigned char* tile = sm.stage[s] + hi0 * 128;
+            const int w0 = first_row(k), w0_next = first_row(k + kProducers);
+            load_chunk(ref_next, 0, k + kProducers);
             // the stage must have been consumed by the MMAs of its previous use
             mbar_wait(&sm.done[(p / kDrainEvery) % kGroups], (uint32_t)(((p / kStages) & 1) ^ 1), abort);
 #pragma unroll
-            for (int rp = 0; rp < MP / 32; ++rp) {
+            for (int j = 0; j < 8; ++j) {
+                if (w0 + j < m) {
+                    uint32_t hw[4], lw[4];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int row = rp * 32 + rq * 8 + j;
-                    if (row < m) {
-                        uint32_t hw[4], lw[4];
-#pragma unroll
-                        for (int pp = 0; pp < 4; ++pp) {
-                            const float v0 = Storage<T>::get(raw[j][pp / (4 / LD)], (2 * pp) % (8 / LD));
-                            const float v1 = Storage<T>::get(raw[j][pp / (4 / LD)], (2 * pp + 1) % (8 / LD));
-                            float r0 = Storage<T>::get(ref[pp / (4 / LD)], (2 * pp) % (8 / LD));
-                            float r1 = Storage<T>::get(ref[pp / (4 / LD)], (2 * pp + 1) % (8 / LD));
-                            if (rp == 0 && j == 0 && rq == 0) r0 = r1 = 0.f;  // operand row 0 carries the reference itself
-                            float x0, x1, l0, l1;
-                            unpk2(sub2(pk2(v0, v1), pk2(r0, r1)), x0, x1);
-                            hw[pp] = pack_bf16x2_rn(x0, x1);
-                            unpk2(sub2(pk2(x0, x1), pk2(__uint_as_float(hw[pp] << 16), __uint_as_float(hw[pp] & 0xffff0000u))),
-                                  l0, l1);
-                            lw[pp] = pack_bf16x2_rn(l0, l1);
-                        }
-                        // this row's registers are free: fetch the same lane's row of the next item into them
-                        if (rp + 1 < MP / 32) {
-                            if (row + 32 < m) load_chunk(raw[j], row + 32, q);
-                        } else {
-                            load_chunk(raw[j], rq * 8 + j, q + kProducers);
-                        }
-                        // operand row `row` (hi) and MP + row (lo); both have the same row & 7
-                        const uint32_t off = (uint32_t)(row * 128 + ((cl ^ (row & 7)) << 4));
-                        *reinterpret_cast<uint4*>(tile + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-                        *reinterpret_cast<uint4*>(tile + MP * 128 + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-                    } else if (MP == 64 && rp == 1 && rq * 8 + j < m) {
-                        // no such row in this item, but the lane's row of the next tile's first item exists
-                        load_chunk(raw[j], rq * 8 + j, q + kProducers);
+                    for (int pp = 0; pp < 4; ++pp) {
+                        const float v0 = Storage<T>::get(raw[j][pp / (4 / LD)], (2 * pp) % (8 / LD));
+                        const float v1 = Storage<T>::get(raw[j][pp / (4 / LD)], (2 * pp + 1) % (8 / LD));
+                        float r0 = Storage<T>::get(ref[pp / (4 / LD)], (2 * pp) % (8 / LD));
+                        float r1 = Storage<T>::get(ref[pp / (4 / LD)], (2 * pp + 1) % (8 / LD));
+                        if (j == 0 && w0 == 0) r0 = r1 = 0.f;  // operand row 0 carries the reference itself
+                        float x0, x1, l0, l1;
+                        unpk2(sub2(pk2(v0, v1), pk2(r0, r1)), x0, x1);
+                        hw[pp] = pack_bf16x2_rn(x0, x1);
+                        unpk2(sub2(pk2(x0, x1), pk2(__uint_as_float(hw[pp] << 16), __uint_as_float(hw[pp] & 0xffff0000u))),
+                              l0, l1);
+                        lw[pp] = pack_bf16x2_rn(l0, l1);
                     }
+                    // this row's registers are free: fetch the same lane's row of the warp's next item into them
+                    if (w0_next + j < m) load_chunk(raw[j], w0_next + j, k + kProducers);
+                    const int orow = rq * 8 + j;  // operand row within the item; orow & 7 == j
+                    const uint32_t off = (uint32_t)(orow * 128 + ((cl ^ j) << 4));
+                    *reinterpret_cast<uint4*>(tile + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                    *reinterpret_cast<uint4*>(tile + MP * 128 + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                } else if (w0_next + j < m) {
+                    // no such Worker in this item, but there is one in the warp's next item
+                    load_chunk(raw[j], w0_next + j, k + kProducers);
                 }
             }
 #pragma unroll
