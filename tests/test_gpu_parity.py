@@ -350,10 +350,14 @@ def test_argument_validation(qn):
 
 # --------------------------------------------------------------------------- tensor-core Gram path (n >= 2^22, m > 8)
 @pytest.mark.parametrize("dtype,m,n,gap", [
-    ("f32", 32, (1 << 22) + 64 * 3 + 4, True),     # config 2's shape class: two tiles per stage, ragged tail
-    ("f32", 9, 1 << 22, True),                     # smallest m on this path: 23 padding rows
-    ("f32", 33, 1 << 22, True),                    # first m with one tile per stage
+    ("f32", 32, (1 << 22) + 64 * 3 + 8, True),     # config 2's shape class: two tiles per stage, ragged tail
+    ("f32", 9, 1 << 22, True),                     # smallest m on this path: four 16-row tiles per stage, 7 padding rows
+    ("f32", 16, (1 << 22) + 8, False),
+    ("f32", 33, 1 << 22, True),                    # first m whose rows are split over a team of two warps
+    ("f32", 64, 1 << 22, True),
     ("bf16", 16, (1 << 22) + 8 * 13, True),
+    ("bf16", 32, 1 << 22, True),
+    ("bf16", 49, 1 << 22, True),                   # team of two warps, the second one with padding rows
     ("bf16", 64, 1 << 22, True),                   # config 4's shape class
     ("bf16", 64, 1 << 22, False),
 ])
