@@ -52,6 +52,8 @@
 // Every wait has an iteration limit:
 // when it runs out the CTA sets an abort flag and an error word, stops waiting, finishes its loops,
 // frees its TMEM and returns; its partial is poisoned with NaN so the solve reports the failure.
+#include <type_traits>
+
 #include "qn_device.cuh"
 
 namespace qn {
@@ -69,7 +71,15 @@ constexpr int kTcWideEvery = 16;                  // drains between fp32 -> fp64
 #define QN_TC_RUN_BYTES 512
 #endif
 constexpr int kTcRunBytes = QN_TC_RUN_BYTES;           // bytes of one row that a CTA's consecutive stages cover
-constexpr int kTcPrefetchAhead = 2;               // a warp prefetches the item this many of its own items ahead into L2
+#ifndef QN_TC_PREFETCH_BF16
+#define QN_TC_PREFETCH_BF16 1
+#endif
+#ifndef QN_TC_PREFETCH_F32
+#define QN_TC_PREFETCH_F32 0
+#endif
+#ifndef QN_TC_FASTPATH_F32
+#define QN_TC_FASTPATH_F32 1
+#endif
 constexpr uint32_t kTcWaitLimit = 1u << 24;       // polls per wait before giving up (each poll may suspend ~1 us)
 
 template <typename T, int MP>
@@ -420,6 +430,9 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
         constexpr int kTeam = Shape::kTeam, kTeams = Shape::kTeams;
         constexpr int kStageChunks = Shape::kStageCols / 8;
         constexpr bool kBf16 = sizeof(T) == 2;
+        // a warp prefetches the item this many of its own items ahead into L2 (measured: helps bf16 storage a
+        // little, costs fp32 storage more than it brings)
+        constexpr int kTcPrefetchAhead = kBf16 ? QN_TC_PREFETCH_BF16 : QN_TC_PREFETCH_F32;
         const int pw = warp < kMmaWarp ? warp : warp == 8 ? 3 : warp - 6;  // warps 0-2, 8, 10-15 -> 0..9
         const int team = pw / kTeam, half = pw % kTeam;
         const int rq = lane / CPI, cl = lane % CPI;
@@ -462,6 +475,18 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
                       "=&r"(raw[j][NW - 3]), "=&r"(raw[j][NW - 2]), "=&r"(raw[j][NW - 1])
                     : "l"(p), "r"((uint32_t)on));
         };
+        // Plain load for items that lie wholly inside the rows (every item but a CTA's last few).
+        auto load_row_plain = [&](int j, const T* p) {
+            if (kBf16)
+                asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                             : "=r"(raw[j][0]), "=r"(raw[j][1]), "=r"(raw[j][2]), "=r"(raw[j][3])
+                             : "l"(p));
+            else
+                asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                             : "=r"(raw[j][0]), "=r"(raw[j][1]), "=r"(raw[j][2]), "=r"(raw[j][3]), "=r"(raw[j][NW - 4]),
+                               "=r"(raw[j][NW - 3]), "=r"(raw[j][NW - 2]), "=r"(raw[j][NW - 1])
+                             : "l"(p));
+        };
         // a warp's part of an item is 64 lines of 128 bytes (its rows x 8 KB / rows): two per lane
         auto prefetch_item = [&](int k) {
             constexpr int kLinesPerRow = Shape::kItemCols * (int)sizeof(T) / 128;
@@ -494,6 +519,9 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
             unsigned char* rows = sm.stage[s] + (tu * RT + w0) * 128;  // operand row of hi(Worker w0)
             const uint32_t xo = (uint32_t)c8 << 4;
             const int64_t col_next = item_col(k + kTeams);
+            // warp-uniform: the whole next item lies inside the rows (then no load needs a predicate)
+            const bool next_inside = (kBf16 || QN_TC_FASTPATH_F32) && kFull && k + kTeams < my_items && item_col0(k + kTeams) + Shape::kItemCols <= n;
+            const T* next_base = g + (int64_t)w0 * n + (next_inside ? col_next : 0);
             if (kTcPrefetchAhead > 0) prefetch_item(k + kTcPrefetchAhead * kTeams);
 
             // ---- the reference of the lane's 8 columns (identical in all lanes and warps that share them)
@@ -578,6 +606,10 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
                         make_uint4(rlo[0], rlo[1], rlo[2], rlo[3]);
             }
 
+            // the row loop, compiled twice: with plain loads of the next item (the common case) and with
+            // predicated ones (the next item is cut by the end of the rows, does not exist, or m < MP)
+            auto convert_rows = [&](auto plain_tag) {
+                constexpr bool kPlain = decltype(plain_tag)::value;
 #pragma unroll
             for (int j = 0; j < RPL; ++j) {
                 {
@@ -600,7 +632,10 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
                         }
                     }
                     // this row's registers are free: fetch the same lane's row of the warp's next item into them
-                    load_row(j, col_next);
+                    if (kPlain)
+                        load_row_plain(j, next_base + (int64_t)j * n);
+                    else
+                        load_row(j, col_next);
                     // operand row w0 + j of the tile; (w0 + j) & 7 == j & 7
                     const uint32_t off = (uint32_t)(j * 128) + (xo ^ (uint32_t)((j & 7) << 4));
                     if (kFull) {
@@ -613,6 +648,11 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
                     }
                 }
             }
+            };
+            if (next_inside)
+                convert_rows(std::true_type{});
+            else
+                convert_rows(std::false_type{});
             // make the generic-proxy stores visible to the tensor core, then hand the warp's part of the item over
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
