@@ -340,13 +340,18 @@ extern "C" qn_status qn_push(qn_handle h, int32_t slot, const void* theta_col, c
     }
     char* trow = static_cast<char*>(h->win_theta) + (size_t)slot * col_bytes;
     char* grow = static_cast<char*>(h->win_g) + (size_t)slot * col_bytes;
-    if (cudaMemcpyAsync(trow, theta_col, col_bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess) s = QN_ERR_CUDA;
-    if (s == QN_OK) {
+    bool theta_landed = false;
+    {
         KernelTimer t(h, st, QN_TIME_ROW);
-        if (qn_launch_row(h->dtype, h->win_g, g_col, grow, h->n, h->m, slot, h->partials, h->max_partials,
-                          h->raw_gram, h->ticket, st, &h->last_launches) != cudaSuccess)
+        if (qn_launch_row(h->dtype, h->win_g, g_col, grow, theta_col, trow, h->n, h->m, slot, h->partials,
+                          h->max_partials, h->raw_gram, h->ticket, h->error_word, &theta_landed, st,
+                          &h->last_launches) != cudaSuccess)
             s = QN_ERR_CUDA;
     }
+    // the register kernel lands only the gradient column
+    if (s == QN_OK && !theta_landed &&
+        cudaMemcpyAsync(trow, theta_col, col_bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        s = QN_ERR_CUDA;
     if (s == QN_OK) h->filled |= (1ull << slot);
     end_call(h);
     return s;
@@ -370,6 +375,7 @@ extern "C" qn_status qn_update_window(qn_handle h, double tau, double lambda, vo
     p.m = h->m;
     p.source = QN_SRC_WINDOW;
     p.raw_gram = h->raw_gram;
+    p.error_word = h->error_word;
     p.tau = tau;
     p.lambda = lambda;
     p.coef = h->coef;

@@ -80,7 +80,6 @@ constexpr int kTcRunBytes = QN_TC_RUN_BYTES;           // bytes of one row that 
 #ifndef QN_TC_FASTPATH_F32
 #define QN_TC_FASTPATH_F32 1
 #endif
-constexpr uint32_t kTcWaitLimit = 1u << 24;       // polls per wait before giving up (each poll may suspend ~1 us)
 
 template <typename T, int MP>
 struct TcShape {
@@ -129,40 +128,6 @@ struct TcSmem {
     // column sums exchanged by the two warps of a team (MP = 64): [team][item parity][warp of the team][chunk]
     alignas(16) uint4 xbuf[MP == 64 ? kTcProducers / 2 : 1][2][2][16][2];
 };
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
-    uint32_t done;
-    asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-        : "=r"(done)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return done != 0;
-}
-// Bounded wait.  Returns false (and raises the abort flag) when the limit runs out or another thread
-// of the CTA has already given up.
-template <bool kBackOff = true>
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
-    if (mbar_try(bar, parity)) return true;  // the common case costs one shared-memory round trip
-    if (*abort) return false;
-    for (uint32_t it = 0; it < kTcWaitLimit; ++it) {
-        if (mbar_try(bar, parity)) return true;
-        // waiting producer and drain warps sleep between polls so that they do not take issue slots from
-        // the MMA warp; the MMA warp itself polls without sleeping
-        if (kBackOff) __nanosleep(64);
-        if ((it & 255u) == 255u && *abort) return false;
-    }
-    *abort = 1;
-    return false;
-}
 
 // K-major, 128-byte swizzle, 8-row groups 1024 bytes apart (the stage built by the producer warps).
 __device__ __forceinline__ uint64_t tc_smem_desc(uint32_t saddr) {

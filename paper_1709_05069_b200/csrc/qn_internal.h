@@ -72,8 +72,11 @@ cudaError_t qn_launch_gram_tc(qn_dtype dtype, const void* g, int64_t n, int m, d
 cudaError_t qn_launch_solve(const qn_solve_params& p, cudaStream_t st, int* launches);
 cudaError_t qn_launch_combine(qn_dtype dtype, const void* theta, const void* g, int64_t n, int m,
                               const qn_coef_block* coef, void* theta_new, cudaStream_t st, int* launches);
-cudaError_t qn_launch_row(qn_dtype dtype, const void* window_g, const void* g_col, void* window_row_out, int64_t n,
-                          int m, int slot, double* partials, int max_partials, double* raw_gram, unsigned int* ticket,
+// Row refresh of the asynchronous window.  Lands g_col in window_row_out; if it can also land theta_col in
+// theta_row_out (bulk-copy kernel) it sets *theta_landed, otherwise the caller copies that column itself.
+cudaError_t qn_launch_row(qn_dtype dtype, const void* window_g, const void* g_col, void* window_row_out,
+                          const void* theta_col, void* theta_row_out, int64_t n, int m, int slot, double* partials,
+                          int max_partials, double* raw_gram, unsigned int* ticket, int* error_word, bool* theta_landed,
                           cudaStream_t st, int* launches);
 cudaError_t qn_solve_init();
 

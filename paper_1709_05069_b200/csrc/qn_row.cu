@@ -12,6 +12,13 @@
 // what bounds the precise mode; its rounding errors are unbiased and average out as 1/sqrt(n).
 // The last CTA to finish adds the per-CTA partial rows in a fixed order and patches row and column
 // `slot` of the Gram: no CTA ever waits for another.
+//
+// Two kernels.  row_kernel keeps its rows in registers (any alignment, both arithmetic modes).  For rows on
+// 16-byte boundaries and n >= QN_PRECISE_BELOW, row_stream_kernel moves the data with bulk copies instead: one
+// thread per CTA issues untiled TMA loads of 4 KB row segments into a ring of shared-memory stages (about
+// 200 KB in flight per SM whatever the occupancy; the register kernel is latency-bound at half the HBM
+// bandwidth), eight warps take the products out of shared memory, and the new gradient and parameter columns
+// are landed in the window by bulk stores straight from the stage, so qn_push needs no separate copy.
 #include "qn_device.cuh"
 
 namespace qn {
@@ -126,12 +133,195 @@ row_kernel(const T* __restrict__ window_g, const T* __restrict__ g_col, T* __res
     }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Bulk-copy variant (fast arithmetic mode, aligned rows).
+// ------------------------------------------------------------------------------------------------
+constexpr int kRsSeg = 4096;      // bytes of one row in a stage: 256 threads x 16 bytes
+constexpr int kRsStages = 5;
+constexpr int kRsConsumers = 256;
+constexpr int kRsThreads = kRsConsumers + 32;  // + one warp whose lane 0 issues the loads
+constexpr int kRsSlots = kRowBlock + 2;        // window rows, the new gradient column, the new parameter column
+
+struct RsSmem {
+    alignas(128) unsigned char seg[kRsStages][kRsSlots][kRsSeg];
+    alignas(8) uint64_t full[kRsStages];
+    uint64_t empty[kRsStages];
+    double red[kRsConsumers / 32][kRowBlock];
+    int abort;
+    int is_last;
+};
+
 template <typename T>
-static cudaError_t launch_row_t(const T* window_g, const T* g_col, T* window_row_out, int64_t n, int m, int slot,
-                                double* partials, int max_partials, double* raw_gram, unsigned int* ticket,
+__global__ void __launch_bounds__(kRsThreads, 1)
+row_stream_kernel(const T* __restrict__ window_g, const T* __restrict__ g_col, T* __restrict__ window_row_out,
+                  const T* __restrict__ theta_col, T* __restrict__ theta_row_out, int64_t n, int m, int slot,
+                  double* __restrict__ partials, double* __restrict__ raw_gram, unsigned int* ticket,
+                  int* __restrict__ error_word) {
+    constexpr int kCols = Storage<T>::kVec;                   // columns per 16-byte vector
+    constexpr int kTileCols = kRsSeg / (int)sizeof(T);        // columns per stage
+    extern __shared__ unsigned char smem_raw[];
+    RsSmem& sm = *reinterpret_cast<RsSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    volatile int* abort = &sm.abort;
+    const int lb = blockIdx.y * kRowBlock;
+    const bool lands = blockIdx.y == 0;  // this slice of rows also lands the new columns in the window
+    const int64_t ntiles = (n + kTileCols - 1) / kTileCols;
+    const int my_tiles = blockIdx.x < ntiles ? (int)((ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x) : 0;
+
+    if (tid == 0) {
+        for (int s = 0; s < kRsStages; ++s) {
+            mbar_init(&sm.full[s], 1);
+            mbar_init(&sm.empty[s], kRsConsumers / 32);
+        }
+        sm.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    double acc[kRowBlock];
+#pragma unroll
+    for (int r = 0; r < kRowBlock; ++r) acc[r] = 0.0;
+
+    if (warp == kRsConsumers / 32) {
+        // ------------------------------------------------------------------ load issue
+        if (lane == 0) {
+            for (int it = 0; it < my_tiles; ++it) {
+                const int s = it % kRsStages, use = it / kRsStages;
+                if (use > 0) mbar_wait(&sm.empty[s], (uint32_t)((use - 1) & 1), abort);
+                const int64_t col0 = (blockIdx.x + (int64_t)it * gridDim.x) * kTileCols;
+                const int64_t left = n - col0;
+                const uint32_t bytes = (uint32_t)((left < kTileCols ? left : kTileCols) * (int64_t)sizeof(T));
+                int nseg = 1 + (lands && theta_col ? 1 : 0);
+#pragma unroll
+                for (int r = 0; r < kRowBlock; ++r) nseg += (lb + r < m && lb + r != slot) ? 1 : 0;
+                mbar_arrive_expect_tx(&sm.full[s], (uint32_t)nseg * bytes);
+#pragma unroll
+                for (int r = 0; r < kRowBlock; ++r)
+                    if (lb + r < m && lb + r != slot)
+                        bulk_load(sm.seg[s][r], window_g + (int64_t)(lb + r) * n + col0, bytes, &sm.full[s]);
+                bulk_load(sm.seg[s][kRowBlock], g_col + col0, bytes, &sm.full[s]);
+                if (lands && theta_col) bulk_load(sm.seg[s][kRowBlock + 1], theta_col + col0, bytes, &sm.full[s]);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ products
+        for (int it = 0; it < my_tiles; ++it) {
+            const int s = it % kRsStages, use = it / kRsStages;
+            const int64_t col0 = (blockIdx.x + (int64_t)it * gridDim.x) * kTileCols;
+            const int64_t left = n - col0;
+            const uint32_t bytes = (uint32_t)((left < kTileCols ? left : kTileCols) * (int64_t)sizeof(T));
+            const bool ok = mbar_wait(&sm.full[s], (uint32_t)(use & 1), abort);
+            if (lands && tid == 0 && ok) {
+                // land the new columns: the stage holds exactly the bytes that go to the window
+                bulk_store(window_row_out + col0, sm.seg[s][kRowBlock], bytes);
+                if (theta_col) bulk_store(theta_row_out + col0, sm.seg[s][kRowBlock + 1], bytes);
+                bulk_store_commit();
+            }
+            const bool live = ok && (uint32_t)(tid * 16) < bytes;  // the last tile may be short; a failed wait adds nothing
+            uint4 xn = make_uint4(0, 0, 0, 0), xl[kRowBlock];
+            if (live) xn = *reinterpret_cast<const uint4*>(sm.seg[s][kRowBlock] + tid * 16);
+#pragma unroll
+            for (int r = 0; r < kRowBlock; ++r) {
+                const int l = lb + r;
+                xl[r] = make_uint4(0, 0, 0, 0);
+                if (l == slot)
+                    xl[r] = xn;
+                else if (live && l < m)
+                    xl[r] = *reinterpret_cast<const uint4*>(sm.seg[s][r] + tid * 16);
+            }
+            float part[kRowBlock];
+#pragma unroll
+            for (int r = 0; r < kRowBlock; ++r) part[r] = 0.f;
+#pragma unroll
+            for (int e = 0; e < kCols; ++e) {
+                const float a = Storage<T>::get(xn, e);
+#pragma unroll
+                for (int r = 0; r < kRowBlock; ++r) part[r] = fmaf(a, Storage<T>::get(xl[r], e), part[r]);
+            }
+#pragma unroll
+            for (int r = 0; r < kRowBlock; ++r) acc[r] += (double)part[r];
+            // the stage may be refilled once every warp has read it and the bulk stores have read it
+            if (lands && tid == 0) bulk_store_wait_read();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.empty[s]);
+        }
+        if (lands && tid == 0) bulk_store_wait_all();  // the landed columns are in global memory before the CTA signals
+    }
+
+    if (*abort) {
+        // a wait ran out: give the bulk copies that may still be in flight into this CTA's shared memory time to
+        // land (bounded: about a millisecond) before the CTA returns
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    }
+    // CTA reduction in a fixed order, then last-CTA-done as in row_kernel
+    if (warp < kRsConsumers / 32) {
+#pragma unroll
+        for (int r = 0; r < kRowBlock; ++r) {
+            const double v = warp_sum(acc[r]);
+            if (lane == 0) sm.red[warp][r] = v;
+        }
+    }
+    __syncthreads();
+    if (tid < kRowBlock && lb + tid < m) {
+        double v = 0.0;
+#pragma unroll
+        for (int w = 0; w < kRsConsumers / 32; ++w) v += sm.red[w][tid];
+        if (*abort) v = __longlong_as_double(0x7ff8000000000000ll);
+        partials[(int64_t)blockIdx.x * m + lb + tid] = v;
+    }
+    if (tid == 0 && *abort && error_word) atomicExch(error_word, 1);
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned int total = gridDim.x * gridDim.y;
+        const unsigned int t = atomicAdd(ticket, 1u);
+        sm.is_last = (t == total - 1);
+    }
+    __syncthreads();
+    if (sm.is_last) {
+        __threadfence();
+        if (tid < m) {
+            double s0 = 0.0, s1 = 0.0;
+            unsigned int p = 0;
+            for (; p + 1 < gridDim.x; p += 2) {
+                s0 += __ldcg(&partials[(int64_t)p * m + tid]);
+                s1 += __ldcg(&partials[(int64_t)(p + 1) * m + tid]);
+            }
+            if (p < gridDim.x) s0 += __ldcg(&partials[(int64_t)p * m + tid]);
+            const double v = s0 + s1;
+            raw_gram[slot * m + tid] = v;
+            raw_gram[tid * m + slot] = v;
+        }
+        if (tid == 0) *ticket = 0;  // ready for the next launch on this stream
+    }
+}
+
+template <typename T>
+static cudaError_t launch_row_t(const T* window_g, const T* g_col, T* window_row_out, const T* theta_col,
+                                T* theta_row_out, int64_t n, int m, int slot, double* partials, int max_partials,
+                                double* raw_gram, unsigned int* ticket, int* error_word, bool* theta_landed,
                                 cudaStream_t st) {
     const bool aligned = (reinterpret_cast<uintptr_t>(window_g) % 16 == 0) &&
                          (reinterpret_cast<uintptr_t>(g_col) % 16 == 0) && ((n * (int64_t)sizeof(T)) % 16 == 0);
+    *theta_landed = false;
+    if (aligned && n >= QN_PRECISE_BELOW && reinterpret_cast<uintptr_t>(window_row_out) % 16 == 0 &&
+        reinterpret_cast<uintptr_t>(theta_col) % 16 == 0 && reinterpret_cast<uintptr_t>(theta_row_out) % 16 == 0) {
+        const int nby = (m + kRowBlock - 1) / kRowBlock;
+        const int64_t ntiles = (n + kRsSeg / (int64_t)sizeof(T) - 1) / (kRsSeg / (int64_t)sizeof(T));
+        int64_t cap = qn_sm_count() / nby;  // one CTA per SM (the stages take most of its shared memory)
+        if (cap < 1) cap = 1;
+        if (cap > max_partials) cap = max_partials;
+        const int gx = (int)(ntiles < cap ? ntiles : cap);
+        auto kern = row_stream_kernel<T>;
+        const size_t smem = sizeof(RsSmem) + 128;
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<dim3(gx, nby), kRsThreads, smem, st>>>(window_g, g_col, window_row_out, theta_col, theta_row_out, n, m,
+                                                     slot, partials, raw_gram, ticket, error_word);
+        *theta_landed = theta_col != nullptr;
+        return cudaGetLastError();
+    }
     const int64_t nitems = aligned ? n / Storage<T>::kVec : n;
     const int nby = (m + kRowBlock - 1) / kRowBlock;
     // one wave of CTAs: every resident slot of every SM gets one CTA (the loop is grid-strided, so a second,
@@ -166,17 +356,20 @@ static cudaError_t launch_row_t(const T* window_g, const T* g_col, T* window_row
 
 }  // namespace qn
 
-cudaError_t qn_launch_row(qn_dtype dtype, const void* window_g, const void* g_col, void* window_row_out, int64_t n,
-                          int m, int slot, double* partials, int max_partials, double* raw_gram, unsigned int* ticket,
+cudaError_t qn_launch_row(qn_dtype dtype, const void* window_g, const void* g_col, void* window_row_out,
+                          const void* theta_col, void* theta_row_out, int64_t n, int m, int slot, double* partials,
+                          int max_partials, double* raw_gram, unsigned int* ticket, int* error_word, bool* theta_landed,
                           cudaStream_t st, int* launches) {
     cudaError_t e =
         dtype == QN_F32
             ? qn::launch_row_t(static_cast<const float*>(window_g), static_cast<const float*>(g_col),
-                               static_cast<float*>(window_row_out), n, m, slot, partials, max_partials, raw_gram,
-                               ticket, st)
+                               static_cast<float*>(window_row_out), static_cast<const float*>(theta_col),
+                               static_cast<float*>(theta_row_out), n, m, slot, partials, max_partials, raw_gram, ticket,
+                               error_word, theta_landed, st)
             : qn::launch_row_t(static_cast<const __nv_bfloat16*>(window_g), static_cast<const __nv_bfloat16*>(g_col),
-                               static_cast<__nv_bfloat16*>(window_row_out), n, m, slot, partials, max_partials,
-                               raw_gram, ticket, st);
+                               static_cast<__nv_bfloat16*>(window_row_out), static_cast<const __nv_bfloat16*>(theta_col),
+                               static_cast<__nv_bfloat16*>(theta_row_out), n, m, slot, partials, max_partials, raw_gram,
+                               ticket, error_word, theta_landed, st);
     if (e == cudaSuccess && launches) *launches += 1;
     return e;
 }

@@ -246,7 +246,12 @@ def test_gram_entry_point(qn, dtype, m, n):
 
 
 # --------------------------------------------------------------------------- asynchronous window
-@pytest.mark.parametrize("dtype,m,n,writes", [("bf16", 8, 120_000, 24), ("f32", 8, 30_001, 12), ("f32", 20, 9_000, 30)])
+@pytest.mark.parametrize("dtype,m,n,writes", [
+    ("bf16", 8, 120_000, 24), ("f32", 8, 30_001, 12), ("f32", 20, 9_000, 30),
+    # n >= 2^22 with aligned rows: the row refresh streams through shared memory with bulk copies (short last
+    # tile; with m = 12 two slices of rows, only one of which lands the new columns)
+    ("bf16", 8, (1 << 22) + 8 * 5, 5), ("f32", 12, (1 << 22) + 4 * 3, 3),
+])
 def test_async_window_matches_sync_oracle(qn, dtype, m, n, writes):
     """Config 3's protocol at reduced n: fill the window, then single-Worker Writes each replacing the oldest
     column with an update after each; every update is compared with the oracle run on the window's contents."""
@@ -280,7 +285,10 @@ def test_async_window_matches_sync_oracle(qn, dtype, m, n, writes):
         assert j1 == j2
         # the last sigma is the square root of round-off (about 1e-8 sigma_1) and differs between the two routes
         np.testing.assert_allclose(s1, s2, rtol=1e-9, atol=1e-6 * s1[0])
-        assert torch.linalg.norm(a.double() - out.double()) <= 1e-6 * torch.linalg.norm(out.double())
+        # below 2^22 columns both routes form every product in fp64; above, the row refresh adds the products of
+        # one work item in fp32, so the two routes differ like two fp32 evaluations (each within 1e-5 of the oracle)
+        bound = 1e-6 if n < (1 << 22) else 2e-5
+        assert torch.linalg.norm(a.double() - out.double()) <= bound * torch.linalg.norm(out.double())
 
 
 def test_async_explicit_slot_and_state(qn):
