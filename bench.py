@@ -47,6 +47,17 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+# DRAM bytes (read + written) per algorithmic byte of one launch, from the ncu captures of small cases summarised
+# under profiles/ (traffic grows in proportion to n: every element is read once per pass).  Keyed by kernel kind,
+# storage type and Gram path; a kernel without a capture of its current form reports no traffic.
+MEASURED_TRAFFIC_RATIO = {
+    ("combine", "f32", "tc"): 0.997,   # combine_vec_kernel<float>, config 2's generator at n = 4,194,304
+    ("gram", "f32", "tc"): 1.007,      # gram_tc_kernel<float, 32>, same capture
+    ("gram", "bf16", "tc"): 1.006,     # gram_tc_kernel<bf16, 64>, config 4's generator at n = 8,388,608
+    ("row", "bf16", "direct"): 0.979,  # row_stream_kernel<bf16>, config 3's generator at n = 33,554,432
+}
+
+
 def algorithmic_bytes(cfg: W.Config):
     """Per update: Gram pass reads m*n, combine reads 2*m*n and writes n elements."""
     b = cfg.elem_bytes
@@ -304,9 +315,11 @@ def main():
     dominant = max(per_kernel, key=lambda k: per_kernel[k][0] * per_kernel[k][1])
     dom_ms = per_kernel[dominant][0]
     achieved = bytes_per[dominant] / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 and bytes_per[dominant] else 0.0
+    ratio = MEASURED_TRAFFIC_RATIO.get((dominant, cfg.dtype, "tc" if cfg.m > 8 else "direct"))
     roofline = {
         "bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
-        "frac": achieved / peak if peak else None, "peak_kind": "of " + peak_kind, "traffic": None,
+        "frac": achieved / peak if peak else None, "peak_kind": "of " + peak_kind,
+        "traffic": ratio * bytes_per[dominant] if ratio else None,
         "algorithmic_bytes_per_launch": bytes_per[dominant], "ms_per_launch": dom_ms,
         "per_kernel_ms": {k: round(v[0], 6) for k, v in per_kernel.items() if v[1]},
         "step_algorithmic_bytes": step_bytes, "step_gbs": step_bytes / (ms_per_step * 1e-3) / 1e9,
