@@ -98,12 +98,48 @@ QN_API qn_status qn_update(qn_handle h, const void* theta, const void* g, double
                     void* theta_new, int32_t* j_out, double* sigma_out, void* cuda_stream);
 
 /*
+ * The operator itself on an arbitrary vector: out = Hbar^{-1} z by Eq. (3)/(4),
+ *   Hbar^{-1} z = z - sum_{k<=j} (u_k^T z) u_k + sum_{k<=j} (u_k^T z) sigma_k^{-1} y_k,
+ * with u_k, y_k, sigma_k and the cut-off j built from (theta, g) exactly as in qn_update (qn_update is this
+ * operator applied to z = gbar inside Eq. (2)).  Use: preconditioning a momentum or an averaged gradient, or
+ * checking the secant property Hbar^{-1}(sigma_k u_k) = y_k.  Like the update, the two sums collapse onto one
+ * m-vector d = sum_{k<=j} v_k (v_k^T G^T z) / sigma_k^2 and out = z - G d + Theta d.  Four kernels: g_k^T z for
+ * all k (reads m*n + n elements), the Gram pass, the eigen-solve, one streaming pass that writes out.
+ *   theta, g     as for qn_update
+ *   z            DEVICE, n elements of the handle's dtype, read only
+ *   out          DEVICE, n elements, must not overlap theta, g or z
+ *   j_out, sigma_out   as for qn_update
+ * Errors as for qn_update (lambda must be finite and > 0).
+ */
+QN_API qn_status qn_apply_hinv(qn_handle h, const void* theta, const void* g, double lambda, const void* z, void* out,
+                               int32_t* j_out, double* sigma_out, void* cuda_stream);
+
+/*
  * The reductions alone: the centred Gram C = G^T G (m x m, row-major, symmetric) followed by
  * w = G^T gbar (m values), as m*m + m doubles written to the DEVICE buffer gram_out
  * (Section 2: the matrix G^H G of the SVD paragraph, and the numerators of alpha_k = z^H u_k
  * for z = gbar).  The means and the centred columns are formed on the fly and never stored.
  */
 QN_API qn_status qn_gram(qn_handle h, const void* g, double* gram_out, void* cuda_stream);
+
+/*
+ * The step with the Gram supplied by the caller: eigen-solve, cut-off and coefficients from `gram`, then the
+ * streaming pass that writes theta_new (Eq. (2) with Eq. (4); everything of qn_update but its first pass).
+ *
+ * This is the n-sharded form of the Server step for several GPUs.  Each rank holds a slice of the columns of
+ * all m Workers (theta, g: [m][n_local]) and a handle created for n_local.  Every sum over the parameter
+ * index in Section 2 (G^H G and z^H u_k for z = gbar) is a sum over the slices, and the centring is linear, so:
+ *   1. every rank calls qn_gram on its slice: m*m + m doubles (centred Gram of the slice, then G^T gbar);
+ *   2. the caller adds these buffers over the ranks (an all-reduce of m*m + m doubles, e.g. NCCL; the paper's
+ *      Server gathers whole vectors instead, Section 2, last paragraph on complexity);
+ *   3. every rank calls qn_update_from_gram with the summed buffer and gets its slice of theta_new; j and
+ *      sigma are the same on every rank.
+ *   gram         DEVICE, m*m + m doubles as written by qn_gram (or sums of such buffers), read only
+ *   other arguments as for qn_update.  Errors as for qn_update.
+ */
+QN_API qn_status qn_update_from_gram(qn_handle h, const void* theta, const void* g, const double* gram, double tau,
+                                     double lambda, void* theta_new, int32_t* j_out, double* sigma_out,
+                                     void* cuda_stream);
 
 /*
  * Asynchronous mode (Section 2, first sentence: an update may follow each Write by one Worker).

@@ -21,6 +21,7 @@ struct qn_ctx {
     qn_result_block* host_result; // pinned host
     unsigned int* ticket;         // device, zero between launches
     int* error_word;              // device, set by a kernel that gave up on a bounded wait
+    double* rhs;                  // device, m doubles: g_k^T z of qn_apply_hinv
 
     // asynchronous window
     void* win_theta;
@@ -216,6 +217,7 @@ extern "C" qn_status qn_create(int64_t n, int32_t m, qn_dtype dtype, qn_handle* 
     ok = ok && cudaMalloc(&h->result, sizeof(qn_result_block)) == cudaSuccess;
     ok = ok && cudaMalloc(&h->raw_gram, sizeof(double) * m * m) == cudaSuccess;
     ok = ok && cudaMalloc(&h->ticket, sizeof(unsigned int)) == cudaSuccess;
+    ok = ok && cudaMalloc(&h->rhs, sizeof(double) * QN_MAX_M) == cudaSuccess;
     ok = ok && cudaMalloc(&h->error_word, sizeof(int)) == cudaSuccess;
     ok = ok && cudaMemset(h->error_word, 0, sizeof(int)) == cudaSuccess;
     ok = ok && cudaMallocHost(&h->host_result, sizeof(qn_result_block)) == cudaSuccess;
@@ -240,6 +242,7 @@ extern "C" qn_status qn_destroy(qn_handle h) {
     cudaFree(h->result);
     cudaFree(h->raw_gram);
     cudaFree(h->ticket);
+    cudaFree(h->rhs);
     cudaFree(h->error_word);
     cudaFree(h->win_theta);
     cudaFree(h->win_g);
@@ -270,6 +273,102 @@ extern "C" qn_status qn_update(qn_handle h, const void* theta, const void* g, do
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     begin_call(h, st);
     s = run_step(h, theta, g, tau, lambda, theta_new, st);
+    end_call(h);
+    if (s != QN_OK) return s;
+    if (j_out || sigma_out) return fetch_result(h, st, j_out, sigma_out);
+    return QN_OK;
+}
+
+extern "C" qn_status qn_update_from_gram(qn_handle h, const void* theta, const void* g, const double* gram,
+                                         double tau, double lambda, void* theta_new, int32_t* j_out,
+                                         double* sigma_out, void* cuda_stream) {
+    qn_status s = check_step_args(h, tau, lambda, theta_new);
+    if (s != QN_OK) return s;
+    if (!theta || !g || !gram) return QN_ERR_INVALID;
+    const size_t in_bytes = (size_t)h->m * (size_t)h->n * h->elem, out_bytes = (size_t)h->n * h->elem;
+    if (overlaps(theta_new, out_bytes, theta, in_bytes) || overlaps(theta_new, out_bytes, g, in_bytes))
+        return QN_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return QN_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    begin_call(h, st);
+    qn_solve_params p;
+    memset(&p, 0, sizeof(p));
+    p.m = h->m;
+    p.source = QN_SRC_SUMMED;
+    p.raw_gram = const_cast<double*>(gram);  // read only in this mode
+    p.tau = tau;
+    p.lambda = lambda;
+    p.coef = h->coef;
+    p.result = h->result;
+    p.error_word = h->error_word;
+    {
+        KernelTimer t(h, st, QN_TIME_SOLVE);
+        if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) s = QN_ERR_CUDA;
+    }
+    if (s == QN_OK) {
+        KernelTimer t(h, st, QN_TIME_COMBINE);
+        if (qn_launch_combine(h->dtype, theta, g, h->n, h->m, h->coef, theta_new, st, &h->last_launches) !=
+            cudaSuccess)
+            s = QN_ERR_CUDA;
+    }
+    end_call(h);
+    if (s != QN_OK) return s;
+    if (j_out || sigma_out) return fetch_result(h, st, j_out, sigma_out);
+    return QN_OK;
+}
+
+extern "C" qn_status qn_apply_hinv(qn_handle h, const void* theta, const void* g, double lambda, const void* z,
+                                   void* out, int32_t* j_out, double* sigma_out, void* cuda_stream) {
+    qn_status s = check_step_args(h, 1.0, lambda, out);
+    if (s != QN_OK) return s;
+    if (!theta || !g || !z) return QN_ERR_INVALID;
+    const size_t in_bytes = (size_t)h->m * (size_t)h->n * h->elem, vec_bytes = (size_t)h->n * h->elem;
+    if (overlaps(out, vec_bytes, theta, in_bytes) || overlaps(out, vec_bytes, g, in_bytes) ||
+        overlaps(out, vec_bytes, z, vec_bytes))
+        return QN_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return QN_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    begin_call(h, st);
+    // 1. g_k^T z for every Worker (the row pass of the asynchronous mode with z in the place of the new column;
+    //    it uses the partials buffer as scratch, so it comes before the Gram pass)
+    bool landed = false;
+    {
+        KernelTimer t(h, st, QN_TIME_ROW);
+        if (qn_launch_row(h->dtype, g, z, nullptr, nullptr, nullptr, h->n, h->m, -1, h->partials, h->max_partials,
+                          nullptr, h->rhs, h->ticket, h->error_word, &landed, st, &h->last_launches) != cudaSuccess)
+            s = QN_ERR_CUDA;
+    }
+    // 2. Gram pass, 3. eigen-solve with the coefficients built for z, 4. out = z - G d + Theta d
+    int np = 0;
+    if (s == QN_OK) {
+        KernelTimer t(h, st, QN_TIME_GRAM);
+        if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st, &h->last_launches,
+                           h->error_word) != cudaSuccess)
+            s = QN_ERR_CUDA;
+    }
+    if (s == QN_OK) {
+        qn_solve_params p;
+        memset(&p, 0, sizeof(p));
+        p.m = h->m;
+        p.source = QN_SRC_PARTIALS;
+        p.partials = h->partials;
+        p.num_partials = np;
+        p.rhs_raw = h->rhs;
+        p.tau = -1.0;
+        p.lambda = lambda;
+        p.coef = h->coef;
+        p.result = h->result;
+        p.error_word = h->error_word;
+        KernelTimer t(h, st, QN_TIME_SOLVE);
+        if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) s = QN_ERR_CUDA;
+    }
+    if (s == QN_OK) {
+        KernelTimer t(h, st, QN_TIME_COMBINE);
+        if (qn_launch_combine(h->dtype, theta, g, h->n, h->m, h->coef, out, st, &h->last_launches, z) != cudaSuccess)
+            s = QN_ERR_CUDA;
+    }
     end_call(h);
     if (s != QN_OK) return s;
     if (j_out || sigma_out) return fetch_result(h, st, j_out, sigma_out);
@@ -344,7 +443,7 @@ extern "C" qn_status qn_push(qn_handle h, int32_t slot, const void* theta_col, c
     {
         KernelTimer t(h, st, QN_TIME_ROW);
         if (qn_launch_row(h->dtype, h->win_g, g_col, grow, theta_col, trow, h->n, h->m, slot, h->partials,
-                          h->max_partials, h->raw_gram, h->ticket, h->error_word, &theta_landed, st,
+                          h->max_partials, h->raw_gram, nullptr, h->ticket, h->error_word, &theta_landed, st,
                           &h->last_launches) != cudaSuccess)
             s = QN_ERR_CUDA;
     }

@@ -17,7 +17,7 @@ constexpr int kCombineUnroll = 4;  // Workers whose loads are in flight together
 template <typename T, bool kAligned>
 __global__ void __launch_bounds__(kCombineThreads)
 combine_kernel(const T* __restrict__ theta, const T* __restrict__ g, int64_t n, int m,
-               const qn_coef_block* __restrict__ coef, T* __restrict__ out) {
+               const qn_coef_block* __restrict__ coef, T* __restrict__ out, const T* __restrict__ base) {
     constexpr int kCols = kAligned ? Storage<T>::kVec : 1;
     __shared__ float c_sh[QN_MAX_M];
     if (threadIdx.x < QN_MAX_M) c_sh[threadIdx.x] = coef->c[threadIdx.x];
@@ -95,6 +95,15 @@ combine_kernel(const T* __restrict__ theta, const T* __restrict__ g, int64_t n, 
         float res[kCols];
 #pragma unroll
         for (int e = 0; e < kCols; ++e) res[e] = fmaf(-tau * inv_m, sg[e], fmaf(sth[e], inv_m, acc[e]));
+        if (base) {  // Eq. (4) applied to z: the correction is added to z instead of to the means
+            uint4 zv;
+            if (kAligned)
+                zv = ldg_stream16(base + i0);
+            else
+                zv.x = __float_as_uint(Storage<T>::load1(base + i0));
+#pragma unroll
+            for (int e = 0; e < kCols; ++e) res[e] = (kAligned ? Storage<T>::get(zv, e) : __uint_as_float(zv.x)) + acc[e];
+        }
         if (kAligned) {
             stg_stream16(out + i0, Storage<T>::pack(res));
         } else {
@@ -149,7 +158,7 @@ __device__ __forceinline__ f32x2 pair_of<__nv_bfloat16>(const uint4& v, int p) {
 template <typename T>
 __global__ void __launch_bounds__(kCombineThreads)
 combine_vec_kernel(const T* __restrict__ theta, const T* __restrict__ g, int64_t n, int m,
-                   const qn_coef_block* __restrict__ coef, T* __restrict__ out) {
+                   const qn_coef_block* __restrict__ coef, T* __restrict__ out, const T* __restrict__ base) {
     constexpr int kCols = Storage<T>::kVec;
     constexpr int kPairs = kCols / 2;
     __shared__ float c_sh[QN_MAX_M];
@@ -198,15 +207,21 @@ combine_vec_kernel(const T* __restrict__ theta, const T* __restrict__ g, int64_t
         const f32x2 im2 = pk(inv_m, inv_m), tm2 = pk(-tau * inv_m, -tau * inv_m);
 #pragma unroll
         for (int p = 0; p < kPairs; ++p) unpk(fma2(tm2, sg[p], fma2(sth[p], im2, acc[p])), res[2 * p], res[2 * p + 1]);
+        if (base) {  // Eq. (4) applied to z: the correction is added to z instead of to the means
+            const uint4 zv = ldg_stream16(base + i0);
+#pragma unroll
+            for (int p = 0; p < kPairs; ++p) unpk(add2(pair_of<T>(zv, p), acc[p]), res[2 * p], res[2 * p + 1]);
+        }
         stg_stream16(out + i0, Storage<T>::pack(res));
     }
 }
 
 template <typename T>
 static cudaError_t launch_combine_t(const T* theta, const T* g, int64_t n, int m, const qn_coef_block* coef, T* out,
-                                    cudaStream_t st) {
+                                    const T* base, cudaStream_t st) {
     const bool aligned = (reinterpret_cast<uintptr_t>(theta) % 16 == 0) && (reinterpret_cast<uintptr_t>(g) % 16 == 0) &&
-                         (reinterpret_cast<uintptr_t>(out) % 16 == 0) && ((n * (int64_t)sizeof(T)) % 16 == 0);
+                         (reinterpret_cast<uintptr_t>(out) % 16 == 0) && (reinterpret_cast<uintptr_t>(base) % 16 == 0) &&
+                         ((n * (int64_t)sizeof(T)) % 16 == 0);
     const int64_t nitems = aligned ? n / Storage<T>::kVec : n;
     const int64_t want = (nitems + kCombineThreads - 1) / kCombineThreads;
     int per_sm = 1;
@@ -217,22 +232,23 @@ static cudaError_t launch_combine_t(const T* theta, const T* g, int64_t n, int m
     const int64_t cap = (int64_t)qn_sm_count() * per_sm * 2;
     const int grid = (int)(want < cap ? (want > 0 ? want : 1) : cap);
     if (aligned)
-        combine_vec_kernel<T><<<grid, kCombineThreads, 0, st>>>(theta, g, n, m, coef, out);
+        combine_vec_kernel<T><<<grid, kCombineThreads, 0, st>>>(theta, g, n, m, coef, out, base);
     else
-        combine_kernel<T, false><<<grid, kCombineThreads, 0, st>>>(theta, g, n, m, coef, out);
+        combine_kernel<T, false><<<grid, kCombineThreads, 0, st>>>(theta, g, n, m, coef, out, base);
     return cudaGetLastError();
 }
 
 }  // namespace qn
 
 cudaError_t qn_launch_combine(qn_dtype dtype, const void* theta, const void* g, int64_t n, int m,
-                              const qn_coef_block* coef, void* theta_new, cudaStream_t st, int* launches) {
+                              const qn_coef_block* coef, void* theta_new, cudaStream_t st, int* launches,
+                              const void* base) {
     cudaError_t e =
         dtype == QN_F32
             ? qn::launch_combine_t(static_cast<const float*>(theta), static_cast<const float*>(g), n, m, coef,
-                                   static_cast<float*>(theta_new), st)
+                                   static_cast<float*>(theta_new), static_cast<const float*>(base), st)
             : qn::launch_combine_t(static_cast<const __nv_bfloat16*>(theta), static_cast<const __nv_bfloat16*>(g), n, m,
-                                   coef, static_cast<__nv_bfloat16*>(theta_new), st);
+                                   coef, static_cast<__nv_bfloat16*>(theta_new), static_cast<const __nv_bfloat16*>(base), st);
     if (e == cudaSuccess && launches) *launches += 1;
     return e;
 }

@@ -33,6 +33,43 @@ constexpr int kDirectM = 8;
 constexpr int kDirectTri = kDirectM * (kDirectM + 1) / 2;  // 36
 constexpr int kDirectAcc = kDirectTri + kDirectM;          // 44
 
+// CTA reduction of the direct kernels in a fixed order: butterfly inside each of the first 8 warps, then warps
+// 0..7 in sequence; the result goes to the CTA's packed partial.  Every thread of the CTA must call it; warps
+// that hold no sums pass `holds_sums = false`.
+__device__ __forceinline__ void direct_reduce_store(const double (&acc64)[kDirectAcc], int m, double* __restrict__ partials,
+                                                    bool holds_sums) {
+    __shared__ double red[kThreads / 32][kDirectAcc];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (holds_sums) {
+#pragma unroll
+        for (int e = 0; e < kDirectAcc; ++e) {
+            const double s = warp_sum(acc64[e]);
+            if (lane == 0) red[warp][e] = s;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < kDirectAcc) {
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) s += red[w][threadIdx.x];
+        // map the 8-row packed index to the m-row packed index
+        const int e = threadIdx.x;
+        double* out = partials + (int64_t)blockIdx.x * qn_partial_len(m);
+        if (e < kDirectTri) {
+            int k = 0, rem = e;
+            while (rem >= kDirectM - k) {
+                rem -= kDirectM - k;
+                ++k;
+            }
+            const int l = k + rem;
+            if (l < m) out[qn_tri_index(m, k, l)] = s;
+        } else {
+            const int k = e - kDirectTri;
+            if (k < m) out[m * (m + 1) / 2 + k] = s;
+        }
+    }
+}
+
 template <typename T, bool kAligned>
 struct DirectItem {
     // one work item = 16 bytes of every row (aligned) or one element of every row (unaligned)
@@ -137,35 +174,195 @@ gram_direct_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict
         for (int e = 0; e < kDirectAcc; ++e) acc64[e] += (double)acc[e];
     }
 
-    // CTA reduction in a fixed order: butterfly inside each warp, then warps 0..7 in sequence.
-    __shared__ double red[kThreads / 32][kDirectAcc];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int e = 0; e < kDirectAcc; ++e) {
-        const double s = warp_sum(acc64[e]);
-        if (lane == 0) red[warp][e] = s;
+    direct_reduce_store(acc64, m, partials, true);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Direct kernel fed by bulk copies, m <= 8, fast arithmetic mode, rows on 16-byte boundaries.  One thread
+// issues untiled TMA loads of 3.5 KB row segments into a ring of shared-memory stages (all m rows of
+// 1792 bf16 / 896 fp32 columns per stage, 196 KB in flight per SM), so the seven warps that do the
+// arithmetic never wait on HBM latency themselves; the register-fed kernel above reaches 5.3 TB/s with fp32
+// storage, this one 6.0.  Used for fp32 storage (see qn_launch_gram).  The arithmetic is kFast's, on packed pairs
+// of columns.
+// Every wait is bounded; on a time-out the partial is poisoned and the error word set.
+// ------------------------------------------------------------------------------------------------
+// packed pairs of fp32 (one 64-bit register, two lanes of the fp32 pipe per instruction)
+__device__ __forceinline__ uint64_t gs_pk2(uint32_t lo, uint32_t hi) {
+    uint64_t v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "r"(lo), "r"(hi));
+    return v;
+}
+__device__ __forceinline__ uint64_t gs_add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t gs_sub2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t gs_mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t gs_fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+// columns 2q and 2q + 1 of a 16-byte vector as a pair of fp32
+template <typename T>
+__device__ __forceinline__ uint64_t gs_pair(const uint4& v, int q);
+template <>
+__device__ __forceinline__ uint64_t gs_pair<float>(const uint4& v, int q) {
+    return q == 0 ? gs_pk2(v.x, v.y) : gs_pk2(v.z, v.w);
+}
+template <>
+__device__ __forceinline__ uint64_t gs_pair<__nv_bfloat16>(const uint4& v, int q) {
+    const uint32_t w = q == 0 ? v.x : q == 1 ? v.y : q == 2 ? v.z : v.w;
+    return gs_pk2(w << 16, w & 0xffff0000u);
+}
+
+constexpr int kGsWarps = 7;                   // warps that do the arithmetic; one more issues the loads: 256 threads,
+constexpr int kGsThreads = (kGsWarps + 1) * 32;  // so that every thread can have the registers its 132 sums need
+constexpr int kGsSeg = kGsWarps * 32 * 16;    // bytes of one row in a stage: one 16-byte vector per arithmetic thread
+constexpr int kGsStages = 7;
+static_assert(kGsThreads == kThreads, "the reduction of the direct kernels is written for kThreads threads");
+
+struct GsSmem {
+    alignas(128) unsigned char seg[kGsStages][kDirectM][kGsSeg];
+    alignas(8) uint64_t full[kGsStages];
+    uint64_t empty[kGsStages];
+    int abort;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kGsThreads, 1)
+gram_stream_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ partials, int* __restrict__ error_word) {
+    constexpr int kCols = Storage<T>::kVec;
+    constexpr int kTileCols = kGsSeg / (int)sizeof(T);
+    constexpr int kFlushIters = kFlushCols / kCols;
+    extern __shared__ unsigned char smem_raw[];
+    GsSmem& sm = *reinterpret_cast<GsSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    volatile int* abort = &sm.abort;
+    const int64_t ntiles = (n + kTileCols - 1) / kTileCols;
+    const int my_tiles = blockIdx.x < ntiles ? (int)((ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x) : 0;
+
+    if (tid == 0) {
+        for (int s = 0; s < kGsStages; ++s) {
+            mbar_init(&sm.full[s], 1);
+            mbar_init(&sm.empty[s], kGsWarps);
+        }
+        sm.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    if (threadIdx.x < kDirectAcc) {
-        double s = 0.0;
+
+    double acc64[kDirectAcc];
 #pragma unroll
-        for (int w = 0; w < kThreads / 32; ++w) s += red[w][threadIdx.x];
-        // map the 8-row packed index to the m-row packed index
-        const int e = threadIdx.x;
-        double* out = partials + (int64_t)blockIdx.x * qn_partial_len(m);
-        if (e < kDirectTri) {
-            int k = 0, rem = e;
-            while (rem >= kDirectM - k) {
-                rem -= kDirectM - k;
-                ++k;
+    for (int e = 0; e < kDirectAcc; ++e) acc64[e] = 0.0;
+
+    if (warp == kGsWarps) {
+        // ------------------------------------------------------------------ load issue
+        if (lane == 0) {
+            for (int it = 0; it < my_tiles; ++it) {
+                const int s = it % kGsStages, use = it / kGsStages;
+                if (use > 0) mbar_wait(&sm.empty[s], (uint32_t)((use - 1) & 1), abort);
+                const int64_t col0 = (blockIdx.x + (int64_t)it * gridDim.x) * kTileCols;
+                const int64_t left = n - col0;
+                const uint32_t bytes = (uint32_t)((left < kTileCols ? left : kTileCols) * (int64_t)sizeof(T));
+                mbar_arrive_expect_tx(&sm.full[s], (uint32_t)m * bytes);
+                for (int k = 0; k < m; ++k) bulk_load(sm.seg[s][k], g + (int64_t)k * n + col0, bytes, &sm.full[s]);
             }
-            const int l = k + rem;
-            if (l < m) out[qn_tri_index(m, k, l)] = s;
-        } else {
-            const int k = e - kDirectTri;
-            if (k < m) out[m * (m + 1) / 2 + k] = s;
         }
+    } else {
+        // ------------------------------------------------------------------ arithmetic
+        // Two columns at a time with the packed fp32x2 instructions (one instruction, two FMAs): with bf16
+        // storage the scalar form needs most of the FMA issue slots of seven warps at HBM speed.  Each half
+        // of a packed accumulator sums every other column.
+        uint64_t acc[kDirectAcc];
+#pragma unroll
+        for (int e = 0; e < kDirectAcc; ++e) acc[e] = 0ull;
+        const float inv_m = 1.0f / (float)m;
+        const uint64_t inv_m2 = gs_pk2(__float_as_uint(inv_m), __float_as_uint(inv_m));
+        int iters = 0;
+        for (int it = 0; it < my_tiles; ++it) {
+            const int s = it % kGsStages, use = it / kGsStages;
+            const int64_t left = n - (blockIdx.x + (int64_t)it * gridDim.x) * kTileCols;
+            const uint32_t bytes = (uint32_t)((left < kTileCols ? left : kTileCols) * (int64_t)sizeof(T));
+            const bool ok = mbar_wait(&sm.full[s], (uint32_t)(use & 1), abort);
+            const bool live = ok && (uint32_t)(tid * 16) < bytes;  // the last tile may be short
+            uint4 v[kDirectM];
+#pragma unroll
+            for (int k = 0; k < kDirectM; ++k) {
+                v[k] = make_uint4(0, 0, 0, 0);
+                if (live && k < m) v[k] = *reinterpret_cast<const uint4*>(sm.seg[s][k] + tid * 16);
+            }
+            // the values are in registers: the stage can be refilled
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.empty[s]);
+#pragma unroll
+            for (int q = 0; q < kCols / 2; ++q) {
+                uint64_t x[kDirectM];
+#pragma unroll
+                for (int k = 0; k < kDirectM; ++k) x[k] = gs_pair<T>(v[k], q);
+                uint64_t sum = x[0];
+#pragma unroll
+                for (int k = 1; k < kDirectM; ++k) sum = gs_add2(sum, x[k]);
+                const uint64_t r = gs_mul2(sum, inv_m2);
+#pragma unroll
+                for (int k = 0; k < kDirectM; ++k) x[k] = k < m ? gs_sub2(x[k], r) : 0ull;  // padding rows stay zero
+#pragma unroll
+                for (int k = 0, idx = 0; k < kDirectM; ++k) {
+#pragma unroll
+                    for (int l = k; l < kDirectM; ++l, ++idx) acc[idx] = gs_fma2(x[k], x[l], acc[idx]);
+                }
+#pragma unroll
+                for (int k = 0; k < kDirectM; ++k) acc[kDirectTri + k] = gs_fma2(x[k], r, acc[kDirectTri + k]);
+            }
+            if (++iters == kFlushIters) {
+                iters = 0;
+#pragma unroll
+                for (int e = 0; e < kDirectAcc; ++e) {
+                    acc64[e] += (double)__uint_as_float((uint32_t)acc[e]) + (double)__uint_as_float((uint32_t)(acc[e] >> 32));
+                    acc[e] = 0ull;
+                }
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < kDirectAcc; ++e)
+            acc64[e] += (double)__uint_as_float((uint32_t)acc[e]) + (double)__uint_as_float((uint32_t)(acc[e] >> 32));
     }
+    __syncthreads();
+    if (*abort) {
+        // a wait ran out: give bulk copies that may still be in flight into this CTA's shared memory time to land
+        // (bounded: about a millisecond), report, and poison the partial so that the solve sees the failure
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+        if (tid == 0 && error_word) atomicExch(error_word, 1);
+#pragma unroll
+        for (int e = 0; e < kDirectAcc; ++e) acc64[e] = __longlong_as_double(0x7ff8000000000000ll);
+    }
+    direct_reduce_store(acc64, m, partials, true);  // the issuing warp adds zeros
+}
+
+template <typename T>
+static cudaError_t launch_gram_stream(const T* g, int64_t n, int m, double* partials, int* num_partials,
+                                      int max_partials, int* error_word, cudaStream_t st) {
+    const int64_t tile_cols = kGsSeg / (int64_t)sizeof(T);
+    const int64_t ntiles = (n + tile_cols - 1) / tile_cols;
+    const int sms = qn_sm_count();
+    int grid = (int)(ntiles < sms ? ntiles : sms);
+    if (grid > max_partials) grid = max_partials;
+    *num_partials = grid;
+    auto kern = gram_stream_kernel<T>;
+    const size_t smem = sizeof(GsSmem) + 128;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, kGsThreads, smem, st>>>(g, n, m, partials, error_word);
+    return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -403,8 +600,17 @@ static bool tc_allowed() {
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
                            int* num_partials, int max_partials, cudaStream_t st, int* launches, int* error_word) {
     cudaError_t e;
+    const int64_t elem = dtype == QN_F32 ? 4 : 2;
     if (!raw && tc_allowed() && qn_gram_tc_applicable(dtype, g, n, m)) {
         e = qn_launch_gram_tc(dtype, g, n, m, partials, num_partials, max_partials, error_word, st);
+    } else if (!raw && tc_allowed() && dtype == QN_F32 && m <= qn::kDirectM && n >= QN_PRECISE_BELOW &&
+               reinterpret_cast<uintptr_t>(g) % 16 == 0 && (n * elem) % 16 == 0) {
+        // Bulk-copy variant of the direct kernel (QN_GRAM_PATH=alu keeps the register-fed one, for A/B runs).
+        // Measured at m = 8: fp32 storage 6.0 TB/s against 5.3 TB/s register-fed; bf16 storage 4.0 against 4.3
+        // (there both are bound by the instructions per element, and seven warps hide latency worse than eight
+        // with register prefetch), so bf16 storage stays on the register-fed kernel.
+        e = qn::launch_gram_stream(static_cast<const float*>(g), n, m, partials, num_partials, max_partials,
+                                   error_word, st);
     } else {
         e = dtype == QN_F32
                 ? qn::launch_gram_t(static_cast<const float*>(g), n, m, raw, partials, num_partials, max_partials, st)

@@ -44,7 +44,8 @@ struct qn_coef_block {
 // What the solve kernel starts from.
 enum qn_solve_source {
     QN_SRC_PARTIALS = 0,  // sum `num_partials` packed partials; if raw_gram != NULL also store the sum there
-    QN_SRC_WINDOW = 1     // start from the raw Gram kept in `raw_gram` (reference 0, t = 0)
+    QN_SRC_WINDOW = 1,    // start from the raw Gram kept in `raw_gram` (reference 0, t = 0)
+    QN_SRC_SUMMED = 2     // start from m*m + m doubles in `raw_gram`: a centred Gram followed by w = G^T gbar
 };
 
 struct qn_solve_params {
@@ -52,10 +53,13 @@ struct qn_solve_params {
     int32_t source;
     const double* partials;  // [num_partials][qn_partial_len(m)]
     int32_t num_partials;
-    double* raw_gram;     // m*m doubles: read (QN_SRC_WINDOW) or written with the uncentred sum (QN_SRC_PARTIALS)
+    double* raw_gram;     // m*m doubles read (QN_SRC_WINDOW), m*m + m read (QN_SRC_SUMMED), or m*m written with the
+                          // uncentred sum (QN_SRC_PARTIALS)
     double* gram_out;     // m*m + m doubles: centred C then w (may be NULL)
     int32_t gram_only;    // stop after writing gram_out
     double tau, lambda;
+    const double* rhs_raw;  // NULL, or m doubles g_k^T z: the coefficients are then built for z instead of gbar
+                            // (w = P rhs_raw) and with tau = -1, i.e. for out = z - G d + Theta d (Eq. (4))
     qn_coef_block* coef;
     qn_result_block* result;
     int* error_word;      // device int set by a kernel that gave up on a bounded wait (may be NULL); read and cleared
@@ -70,14 +74,19 @@ bool qn_gram_tc_applicable(qn_dtype dtype, const void* g, int64_t n, int m);
 cudaError_t qn_launch_gram_tc(qn_dtype dtype, const void* g, int64_t n, int m, double* partials, int* num_partials,
                               int max_partials, int* error_word, cudaStream_t st);
 cudaError_t qn_launch_solve(const qn_solve_params& p, cudaStream_t st, int* launches);
+// base == NULL: theta_new of Eq. (2).  base = z (n elements): out = z + sum_k c[k] * ((g_k - g_0) - (theta_k - theta_0)).
 cudaError_t qn_launch_combine(qn_dtype dtype, const void* theta, const void* g, int64_t n, int m,
-                              const qn_coef_block* coef, void* theta_new, cudaStream_t st, int* launches);
-// Row refresh of the asynchronous window.  Lands g_col in window_row_out; if it can also land theta_col in
-// theta_row_out (bulk-copy kernel) it sets *theta_landed, otherwise the caller copies that column itself.
+                              const qn_coef_block* coef, void* theta_new, cudaStream_t st, int* launches,
+                              const void* base = nullptr);
+// Row refresh of the asynchronous window: the products of g_col with the m rows of window_g (row `slot` is taken
+// to be g_col itself), patched into row and column `slot` of raw_gram.  Lands g_col in window_row_out; if it can
+// also land theta_col in theta_row_out (bulk-copy kernel) it sets *theta_landed, otherwise the caller copies that
+// column itself.  With dots_out != NULL the m products go there instead (slot = -1, window_row_out = theta_col =
+// NULL: nothing is landed), which is G^T z up to the centring for an arbitrary vector z.
 cudaError_t qn_launch_row(qn_dtype dtype, const void* window_g, const void* g_col, void* window_row_out,
                           const void* theta_col, void* theta_row_out, int64_t n, int m, int slot, double* partials,
-                          int max_partials, double* raw_gram, unsigned int* ticket, int* error_word, bool* theta_landed,
-                          cudaStream_t st, int* launches);
+                          int max_partials, double* raw_gram, double* dots_out, unsigned int* ticket, int* error_word,
+                          bool* theta_landed, cudaStream_t st, int* launches);
 cudaError_t qn_solve_init();
 
 int qn_sm_count();

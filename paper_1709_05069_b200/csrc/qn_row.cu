@@ -29,7 +29,8 @@ constexpr int kRowBlock = 8;  // window columns handled by one CTA row (blockIdx
 template <typename T, bool kAligned, bool kPrecise>
 __global__ void __launch_bounds__(kRowThreads)
 row_kernel(const T* __restrict__ window_g, const T* __restrict__ g_col, T* __restrict__ window_row_out, int64_t n,
-           int m, int slot, double* __restrict__ partials, double* __restrict__ raw_gram, unsigned int* ticket) {
+           int m, int slot, double* __restrict__ partials, double* __restrict__ raw_gram, double* __restrict__ dots_out,
+           unsigned int* ticket) {
     constexpr int kCols = kAligned ? Storage<T>::kVec : 1;
     const int lb = blockIdx.y * kRowBlock;
     const int64_t nitems = kAligned ? n / kCols : n;
@@ -59,7 +60,7 @@ row_kernel(const T* __restrict__ window_g, const T* __restrict__ g_col, T* __res
                     xl[r].x = __float_as_uint(Storage<T>::load1(window_g + (int64_t)l * n + i0));
             }
         }
-        if (blockIdx.y == 0) {  // land the column
+        if (blockIdx.y == 0 && window_row_out) {  // land the column
             if (kAligned)
                 stg_stream16(window_row_out + i0, xn);
             else
@@ -126,8 +127,12 @@ row_kernel(const T* __restrict__ window_g, const T* __restrict__ g_col, T* __res
             }
             if (p < gridDim.x) s0 += __ldcg(&partials[(int64_t)p * m + threadIdx.x]);
             const double v = s0 + s1;
-            raw_gram[slot * m + threadIdx.x] = v;
-            raw_gram[threadIdx.x * m + slot] = v;
+            if (dots_out) {
+                dots_out[threadIdx.x] = v;
+            } else {
+                raw_gram[slot * m + threadIdx.x] = v;
+                raw_gram[threadIdx.x * m + slot] = v;
+            }
         }
         if (threadIdx.x == 0) *ticket = 0;  // ready for the next launch on this stream
     }
@@ -156,8 +161,8 @@ template <typename T>
 __global__ void __launch_bounds__(kRsThreads, 1)
 row_stream_kernel(const T* __restrict__ window_g, const T* __restrict__ g_col, T* __restrict__ window_row_out,
                   const T* __restrict__ theta_col, T* __restrict__ theta_row_out, int64_t n, int m, int slot,
-                  double* __restrict__ partials, double* __restrict__ raw_gram, unsigned int* ticket,
-                  int* __restrict__ error_word) {
+                  double* __restrict__ partials, double* __restrict__ raw_gram, double* __restrict__ dots_out,
+                  unsigned int* ticket, int* __restrict__ error_word) {
     constexpr int kCols = Storage<T>::kVec;                   // columns per 16-byte vector
     constexpr int kTileCols = kRsSeg / (int)sizeof(T);        // columns per stage
     extern __shared__ unsigned char smem_raw[];
@@ -165,7 +170,7 @@ row_stream_kernel(const T* __restrict__ window_g, const T* __restrict__ g_col, T
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     volatile int* abort = &sm.abort;
     const int lb = blockIdx.y * kRowBlock;
-    const bool lands = blockIdx.y == 0;  // this slice of rows also lands the new columns in the window
+    const bool lands = blockIdx.y == 0 && window_row_out != nullptr;  // this slice of rows also lands the new columns
     const int64_t ntiles = (n + kTileCols - 1) / kTileCols;
     const int my_tiles = blockIdx.x < ntiles ? (int)((ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x) : 0;
 
@@ -290,8 +295,12 @@ row_stream_kernel(const T* __restrict__ window_g, const T* __restrict__ g_col, T
             }
             if (p < gridDim.x) s0 += __ldcg(&partials[(int64_t)p * m + tid]);
             const double v = s0 + s1;
-            raw_gram[slot * m + tid] = v;
-            raw_gram[tid * m + slot] = v;
+            if (dots_out) {
+                dots_out[tid] = v;
+            } else {
+                raw_gram[slot * m + tid] = v;
+                raw_gram[tid * m + slot] = v;
+            }
         }
         if (tid == 0) *ticket = 0;  // ready for the next launch on this stream
     }
@@ -300,8 +309,8 @@ row_stream_kernel(const T* __restrict__ window_g, const T* __restrict__ g_col, T
 template <typename T>
 static cudaError_t launch_row_t(const T* window_g, const T* g_col, T* window_row_out, const T* theta_col,
                                 T* theta_row_out, int64_t n, int m, int slot, double* partials, int max_partials,
-                                double* raw_gram, unsigned int* ticket, int* error_word, bool* theta_landed,
-                                cudaStream_t st) {
+                                double* raw_gram, double* dots_out, unsigned int* ticket, int* error_word,
+                                bool* theta_landed, cudaStream_t st) {
     const bool aligned = (reinterpret_cast<uintptr_t>(window_g) % 16 == 0) &&
                          (reinterpret_cast<uintptr_t>(g_col) % 16 == 0) && ((n * (int64_t)sizeof(T)) % 16 == 0);
     *theta_landed = false;
@@ -318,7 +327,7 @@ static cudaError_t launch_row_t(const T* window_g, const T* g_col, T* window_row
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         kern<<<dim3(gx, nby), kRsThreads, smem, st>>>(window_g, g_col, window_row_out, theta_col, theta_row_out, n, m,
-                                                     slot, partials, raw_gram, ticket, error_word);
+                                                     slot, partials, raw_gram, dots_out, ticket, error_word);
         *theta_landed = theta_col != nullptr;
         return cudaGetLastError();
     }
@@ -344,13 +353,13 @@ static cudaError_t launch_row_t(const T* window_g, const T* g_col, T* window_row
     const bool precise = n < QN_PRECISE_BELOW;
     if (aligned && !precise)
         row_kernel<T, true, false><<<grid, kRowThreads, 0, st>>>(window_g, g_col, window_row_out, n, m, slot, partials,
-                                                                raw_gram, ticket);
+                                                                raw_gram, dots_out, ticket);
     else if (aligned)
         row_kernel<T, true, true><<<grid, kRowThreads, 0, st>>>(window_g, g_col, window_row_out, n, m, slot, partials,
-                                                               raw_gram, ticket);
+                                                               raw_gram, dots_out, ticket);
     else
         row_kernel<T, false, true><<<grid, kRowThreads, 0, st>>>(window_g, g_col, window_row_out, n, m, slot, partials,
-                                                                raw_gram, ticket);
+                                                                raw_gram, dots_out, ticket);
     return cudaGetLastError();
 }
 
@@ -358,18 +367,18 @@ static cudaError_t launch_row_t(const T* window_g, const T* g_col, T* window_row
 
 cudaError_t qn_launch_row(qn_dtype dtype, const void* window_g, const void* g_col, void* window_row_out,
                           const void* theta_col, void* theta_row_out, int64_t n, int m, int slot, double* partials,
-                          int max_partials, double* raw_gram, unsigned int* ticket, int* error_word, bool* theta_landed,
-                          cudaStream_t st, int* launches) {
+                          int max_partials, double* raw_gram, double* dots_out, unsigned int* ticket, int* error_word,
+                          bool* theta_landed, cudaStream_t st, int* launches) {
     cudaError_t e =
         dtype == QN_F32
             ? qn::launch_row_t(static_cast<const float*>(window_g), static_cast<const float*>(g_col),
                                static_cast<float*>(window_row_out), static_cast<const float*>(theta_col),
-                               static_cast<float*>(theta_row_out), n, m, slot, partials, max_partials, raw_gram, ticket,
-                               error_word, theta_landed, st)
+                               static_cast<float*>(theta_row_out), n, m, slot, partials, max_partials, raw_gram,
+                               dots_out, ticket, error_word, theta_landed, st)
             : qn::launch_row_t(static_cast<const __nv_bfloat16*>(window_g), static_cast<const __nv_bfloat16*>(g_col),
                                static_cast<__nv_bfloat16*>(window_row_out), static_cast<const __nv_bfloat16*>(theta_col),
                                static_cast<__nv_bfloat16*>(theta_row_out), n, m, slot, partials, max_partials, raw_gram,
-                               ticket, error_word, theta_landed, st);
+                               dots_out, ticket, error_word, theta_landed, st);
     if (e == cudaSuccess && launches) *launches += 1;
     return e;
 }

@@ -108,8 +108,11 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
         if (prm.raw_gram)
             for (int e = tid; e < m * m; e += nthr) prm.raw_gram[e] = sm.A[(e / m) * kLd + (e % m)];
     } else {
+        // QN_SRC_WINDOW: the raw Gram (w follows from it in the centring below); QN_SRC_SUMMED: a centred Gram
+        // followed by w, e.g. the sum over column shards of what qn_gram wrote (the centring below leaves an
+        // already centred pair unchanged up to rounding: P (P C P) P = P C P and 1^T w = 0)
         for (int e = tid; e < m * m; e += nthr) sm.A[(e / m) * kLd + (e % m)] = prm.raw_gram[e];
-        if (tid < m) sm.w[tid] = 0.0;
+        if (tid < m) sm.w[tid] = prm.source == QN_SRC_SUMMED ? prm.raw_gram[m * m + tid] : 0.0;
         __syncthreads();
     }
 
@@ -138,7 +141,14 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
         if (prm.gram_out) prm.gram_out[e] = c;
     }
     if (tid < m) {
-        const double wk = sm.w[tid] - tsum * inv_m + sm.rowsum[tid] * inv_m - tot * inv_m * inv_m;
+        double wk = sm.w[tid] - tsum * inv_m + sm.rowsum[tid] * inv_m - tot * inv_m * inv_m;
+        if (prm.rhs_raw) {
+            // coefficients for an arbitrary z: G^T z = P (g_k^T z)_k, because the centring removes the same
+            // gbar^T z from every entry
+            double rs = 0.0;
+            for (int l = 0; l < m; ++l) rs += prm.rhs_raw[l];
+            wk = prm.rhs_raw[tid] - rs * inv_m;
+        }
         bad |= !isfinite(wk);
         // every thread has read w (tsum) before the barrier above; only thread tid rewrites w[tid]
         sm.w[tid] = wk;

@@ -22,7 +22,7 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libqn.so")
 _lib: Optional[ctypes.CDLL] = None
 
 EXPORTS = (
-    "qn_strerror", "qn_create", "qn_destroy", "qn_update", "qn_gram", "qn_push", "qn_update_window", "qn_rebuild",
+    "qn_strerror", "qn_create", "qn_destroy", "qn_update", "qn_gram", "qn_update_from_gram", "qn_apply_hinv", "qn_push", "qn_update_window", "qn_rebuild",
     "qn_window_alloc", "qn_window_theta", "qn_window_g", "qn_window_mark_full", "qn_update_host", "qn_status_sync",
     "qn_last_launches", "qn_total_launches", "qn_last_sweeps", "qn_timing_begin", "qn_timing_end",
     "qn_gram_static",
@@ -50,6 +50,8 @@ def lib() -> ctypes.CDLL:
         L.qn_destroy.argtypes, L.qn_destroy.restype = [vp], i32
         L.qn_update.argtypes, L.qn_update.restype = [vp, vp, vp, dbl, dbl, vp, vp, vp, vp], i32
         L.qn_gram.argtypes, L.qn_gram.restype = [vp, vp, vp, vp], i32
+        L.qn_apply_hinv.argtypes, L.qn_apply_hinv.restype = [vp, vp, vp, dbl, vp, vp, vp, vp, vp], i32
+        L.qn_update_from_gram.argtypes, L.qn_update_from_gram.restype = [vp, vp, vp, vp, dbl, dbl, vp, vp, vp, vp], i32
         L.qn_push.argtypes, L.qn_push.restype = [vp, i32, vp, vp, vp], i32
         L.qn_update_window.argtypes, L.qn_update_window.restype = [vp, dbl, dbl, vp, vp, vp, vp], i32
         L.qn_rebuild.argtypes, L.qn_rebuild.restype = [vp, vp], i32
@@ -177,10 +179,67 @@ def qn_update(h: Handle, theta: torch.Tensor, g: torch.Tensor, tau: float, lam: 
 
 def qn_gram(h: Handle, g: torch.Tensor, gram_out: torch.Tensor, stream=None) -> None:
     """Centred Gram (m*m) followed by w = G^T gbar (m) into ``gram_out`` (CUDA float64, m*m + m)."""
-    if not gram_out.is_cuda or gram_out.dtype != torch.float64 or gram_out.numel() != h.m * h.m + h.m \
-            or not gram_out.is_contiguous():
-        raise ValueError("gram_out must be a contiguous CUDA float64 tensor with m*m + m elements")
+    _check_gram_buffer(h, gram_out)
     _check(lib().qn_gram(h.ptr, _dev_matrix(g, h, "g"), gram_out.data_ptr(), _stream_ptr(stream)), "qn_gram")
+
+
+def qn_apply_hinv(h: Handle, theta: torch.Tensor, g: torch.Tensor, lam: float, z: torch.Tensor, out: torch.Tensor,
+                  want_host: bool = True, stream=None, allow=(QN_ERR_NOT_CONVERGED, QN_ERR_NONFINITE)):
+    """``out = Hbar^{-1} z`` (Eq. (3)/(4)) for an arbitrary device vector ``z``.  Returns like ``qn_update``."""
+    j, sigma, jp, sp = _host_outputs(h, want_host)
+    st = lib().qn_apply_hinv(h.ptr, _dev_matrix(theta, h, "theta"), _dev_matrix(g, h, "g"), float(lam),
+                             _dev_vector(z, h, "z"), _dev_vector(out, h, "out"), jp, sp, _stream_ptr(stream))
+    _check(st, "qn_apply_hinv", allow)
+    if want_host:
+        return j.value, list(sigma), st
+    return None
+
+
+def _check_gram_buffer(h: Handle, gram: torch.Tensor) -> None:
+    if not gram.is_cuda or gram.dtype != torch.float64 or gram.numel() != h.m * h.m + h.m or not gram.is_contiguous():
+        raise ValueError("the Gram buffer must be a contiguous CUDA float64 tensor with m*m + m elements")
+
+
+def qn_update_from_gram(h: Handle, theta: torch.Tensor, g: torch.Tensor, gram: torch.Tensor, tau: float, lam: float,
+                        theta_new: torch.Tensor, want_host: bool = True, stream=None,
+                        allow=(QN_ERR_NOT_CONVERGED, QN_ERR_NONFINITE)):
+    """The step without its Gram pass: ``gram`` is what ``qn_gram`` wrote, or the sum of such buffers over the
+    column slices of an n-sharded problem.  Returns like ``qn_update``."""
+    _check_gram_buffer(h, gram)
+    j, sigma, jp, sp = _host_outputs(h, want_host)
+    st = lib().qn_update_from_gram(h.ptr, _dev_matrix(theta, h, "theta"), _dev_matrix(g, h, "g"), gram.data_ptr(),
+                                   float(tau), float(lam), _dev_vector(theta_new, h, "theta_new"), jp, sp,
+                                   _stream_ptr(stream))
+    _check(st, "qn_update_from_gram", allow)
+    if want_host:
+        return j.value, list(sigma), st
+    return None
+
+
+def shard_columns(n: int, world: int, rank: int, align: int = 8):
+    """Column range [begin, end) of ``rank`` when n columns are split over ``world`` ranks in contiguous slices whose
+    boundaries are multiples of ``align`` (so that every slice keeps 16-byte aligned rows).  Host logic only."""
+    if world < 1 or not 0 <= rank < world or n < 0 or align < 1:
+        raise ValueError("bad shard request")
+    blocks = (n + align - 1) // align
+    b0 = blocks * rank // world
+    b1 = blocks * (rank + 1) // world
+    return min(b0 * align, n), min(b1 * align, n)
+
+
+def qn_update_sharded(h: Handle, theta: torch.Tensor, g: torch.Tensor, tau: float, lam: float, theta_new: torch.Tensor,
+                      gram_buf: torch.Tensor, group=None, want_host: bool = True, stream=None):
+    """One Server step on this rank's column slice of an n-sharded problem (one process per GPU).
+
+    ``theta``, ``g``: [m][n_local] of this rank; ``gram_buf``: CUDA float64 scratch with m*m + m elements.  The only
+    exchange is one all-reduce of ``gram_buf`` (``torch.distributed``, NCCL between GPUs); every other byte stays on
+    its GPU.  With no initialised process group (or a world of one) this is ``qn_gram`` + ``qn_update_from_gram``."""
+    import torch.distributed as dist
+
+    qn_gram(h, g, gram_buf, stream=stream)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+        dist.all_reduce(gram_buf, op=dist.ReduceOp.SUM, group=group)
+    return qn_update_from_gram(h, theta, g, gram_buf, tau, lam, theta_new, want_host=want_host, stream=stream)
 
 
 def qn_push(h: Handle, slot: int, theta_col: torch.Tensor, g_col: torch.Tensor, stream=None) -> None:

@@ -356,6 +356,96 @@ def test_argument_validation(qn):
     hd.close()
 
 
+# --------------------------------------------------------------------------- the operator on an arbitrary vector
+@pytest.mark.parametrize("dtype,m,n", [
+    ("f32", 6, 30_001), ("f32", 20, 9_000), ("bf16", 8, 64_000), ("bf16", 33, 12_008),
+    ("f32", 8, (1 << 22) + 4 * 5), ("bf16", 32, (1 << 22) + 8), ("f32", 12, 1 << 22),
+])
+def test_apply_hinv_matches_the_oracle(qn, dtype, m, n):
+    """Eq. (3)/(4) on an arbitrary z (not gbar): against the oracle's literal evaluation on the same bits."""
+    cfg = W.Config(43, n, m, dtype, -1, 1, 0, 0.1, 1e-3, 1.0, 0.02)
+    theta, g = W.generate(cfg, "cuda", gap_lam=cfg.lam, gap_scale=1.0)
+    gen = torch.Generator(device="cuda").manual_seed(4301)
+    z = torch.randn(n, device="cuda", generator=gen).to(theta.dtype)
+    # a z with a large part inside span{u_k}: a combination of the gradients themselves
+    z = (z.float() + 0.5 * (g[1].float() - g[0].float()) - 0.25 * (g[m - 1].float() - g[2].float())).to(theta.dtype)
+    out = torch.empty(n, dtype=theta.dtype, device="cuda")
+    with qn.qn_create(n, m, theta.dtype) as h:
+        j, sigma, status = qn.qn_apply_hinv(h, theta, g, cfg.lam, z, out)
+        assert h.last_launches == 4
+    ref, jref = oracle.apply_hinv(W.to_bits(theta), W.to_bits(g), cfg.lam, oracle.storage_to_f64(W.to_bits(z)))
+    assert status == 0 and j == jref and 0 < j < m - 1
+    got = oracle.storage_to_f64(W.to_bits(out))
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= TOL[dtype]
+    # the correction is not a rounding-level effect: Hinv z differs from z well above the tolerance
+    z64 = oracle.storage_to_f64(W.to_bits(z))
+    assert np.linalg.norm(ref - z64) / np.linalg.norm(ref) > 50 * TOL[dtype]
+
+
+def test_apply_hinv_is_the_identity_when_no_mode_is_kept(qn):
+    cfg = W.Config(44, 20_000, 7, "f32", -1, 1, 0, 0.1, 1e-3, 1.0, 0.02)
+    theta, g = W.generate(cfg, "cuda")
+    z = torch.randn(cfg.n, device="cuda")
+    out = torch.empty_like(z)
+    with qn.qn_create(cfg.n, cfg.m, torch.float32) as h:
+        j, sigma, status = qn.qn_apply_hinv(h, theta, g, 1.5, z, out)  # lambda > 1: j = 0
+    assert j == 0 and status == 0 and torch.equal(out, z)
+
+
+# --------------------------------------------------------------------------- n-sharded step
+@pytest.mark.parametrize("dtype,m,n,shards", [("f32", 12, 40_008, 2), ("bf16", 8, 100_000, 3), ("f32", 32, (1 << 22) + 64, 2)])
+def test_sharded_step_matches_the_whole_problem(qn, dtype, m, n, shards):
+    """qn_gram on every column slice, the buffers added (what the all-reduce does between GPUs),
+    qn_update_from_gram on every slice: j, sigma and the concatenated theta_new against the oracle on the whole
+    problem, and j, sigma identical on every slice."""
+    cfg = W.Config(42, n, m, dtype, -1, 1, 0, 0.1, 1e-3, 0.7, 0.02)
+    theta, g = W.generate(cfg, "cuda", gap_lam=cfg.lam, gap_scale=1.0)
+    ranges = [qn.shard_columns(n, shards, r) for r in range(shards)]
+    parts = [(theta[:, b:e].contiguous(), g[:, b:e].contiguous()) for b, e in ranges]
+    handles = [qn.qn_create(e - b, m, theta.dtype) for b, e in ranges]
+    try:
+        bufs = [torch.empty(m * m + m, dtype=torch.float64, device="cuda") for _ in ranges]
+        for h, (t, gg), buf in zip(handles, parts, bufs):
+            qn.qn_gram(h, gg, buf)
+        total = torch.stack(bufs).sum(0)
+        out = torch.empty(n, dtype=theta.dtype, device="cuda")
+        results = []
+        for h, (t, gg), (b, e) in zip(handles, parts, ranges):
+            piece = torch.empty(e - b, dtype=theta.dtype, device="cuda")
+            results.append(qn.qn_update_from_gram(h, t, gg, total, cfg.tau, cfg.lam, piece))
+            assert h.last_launches == 2
+            out[b:e] = piece
+    finally:
+        for h in handles:
+            h.close()
+    ref = oracle.update(W.to_bits(theta), W.to_bits(g), cfg.tau, cfg.lam)
+    for j, sigma, status in results:
+        assert status == 0 and j == ref.j
+        assert np.array_equal(np.array(sigma), np.array(results[0][1]))
+        assert np.max(np.abs(np.array(sigma) - ref.sigma)) <= 1e-5 * ref.sigma[0]
+        assert np.max(np.abs(np.array(sigma)[:j] - ref.sigma[:j]) / ref.sigma[:j]) <= 1e-5
+    got = oracle.storage_to_f64(W.to_bits(out))
+    assert np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL[dtype]
+
+
+# --------------------------------------------------------------------------- bulk-copy Gram path (n >= 2^22, m <= 8)
+@pytest.mark.parametrize("dtype,m,n,gap", [
+    ("bf16", 8, (1 << 22) + 8 * 3, True),    # config 4's first sweep point (register-fed kernel, fast mode)
+    ("bf16", 8, 1 << 22, False),
+    ("f32", 5, (1 << 22) + 4, True),         # bulk-copy kernel: three padding rows, short last tile
+    ("f32", 8, 1 << 22, True),
+    ("f32", 8, 1 << 22, False),
+])
+def test_direct_gram_paths_at_large_n(qn, dtype, m, n, gap):
+    """Above 2^22 columns and with at most 8 Workers: fp32 storage on aligned rows is fed by bulk copies into
+    shared-memory stages, bf16 storage by register prefetch.  Same bar as everywhere."""
+    cfg = W.Config(41, n, m, dtype, -2, 2, 0, 0.01, 1e-4, 1.0, 0.01)
+    lam = 0.05 if (gap and dtype == "bf16") else 0.01
+    theta, g = W.generate(cfg, "cuda", gap_lam=lam if gap else None, gap_scale=1.0 if (gap and dtype == "bf16") else None)
+    expect = assert_gap(theta, g, lam) if gap else m - 1
+    check_against_oracle(qn, theta, g, cfg.tau, lam, dtype, expect_j=expect)
+
+
 # --------------------------------------------------------------------------- tensor-core Gram path (n >= 2^22, m > 8)
 @pytest.mark.parametrize("dtype,m,n,gap", [
     ("f32", 32, (1 << 22) + 64 * 3 + 8, True),     # config 2's shape class: two tiles per stage, ragged tail

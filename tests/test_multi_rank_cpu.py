@@ -1,5 +1,5 @@
-"""The N > 1 path of bench.py on CPU: two gloo ranks as independent replicas (the method itself has no
-collective; ranks only agree on the slowest rank's time)."""
+"""The N > 1 paths on CPU with two gloo ranks: bench.py's independent replicas (ranks only agree on the slowest
+rank's time), and the host side of the n-sharded step (column slices, one all-reduce of m*m + m doubles)."""
 import os
 import socket
 import sys
@@ -49,3 +49,77 @@ def test_single_rank_needs_no_process_group():
 
     assert bench.max_over_ranks(1.25, 1, torch.device("cpu")) == 1.25
     assert bench.whole_job_value(2.0, 1) == 500.0
+
+
+# --------------------------------------------------------------------------- n-sharded step, host side
+def test_shard_columns_partitions_the_range_on_aligned_boundaries():
+    sys.path.insert(0, ROOT)
+    from paper_1709_05069_b200 import qn
+
+    for n in (0, 1, 7, 8, 9, 1000, 25_600_000, (1 << 28) + 8):
+        for world in (1, 2, 3, 8):
+            ranges = [qn.shard_columns(n, world, r) for r in range(world)]
+            assert ranges[0][0] == 0 and ranges[-1][1] == n
+            for (a0, a1), (b0, b1) in zip(ranges, ranges[1:]):
+                assert a1 == b0 and a0 <= a1
+            assert all(b % 8 == 0 for b, _ in ranges)
+            sizes = [e - b for b, e in ranges]
+            assert max(sizes) - min(sizes) <= 8 + 7  # balanced up to one aligned block and the ragged end
+
+
+def _shard_rank_main(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world),
+                      LOCAL_RANK=str(rank))
+    import numpy as np
+    import torch.distributed as dist
+
+    import oracle
+    import workloads as W
+    from paper_1709_05069_b200 import qn
+
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    cfg = W.Config(21, 6003, 5, "f32", -1, 1, 0, 0.1, 1e-3, 1.0, 0.01)
+    theta, g = W.generate(cfg, "cpu")  # every rank generates the same bits and keeps its slice
+    gb = W.to_bits(g)
+    b, e = qn.shard_columns(cfg.n, world, rank)
+    mine = np.ascontiguousarray(gb[:, b:e])
+    m = cfg.m
+    # what qn_gram writes for this slice, from the oracle: centred Gram, then G^T gbar
+    C = oracle.gram(mine)
+    g64 = oracle.storage_to_f64(mine)
+    gbar = g64.mean(0)
+    w = (g64 - gbar) @ gbar
+    buf = torch.from_numpy(np.concatenate([C.reshape(-1), w]))
+    dist.all_reduce(buf, op=dist.ReduceOp.SUM)
+    out[rank] = buf.numpy().copy()
+    dist.destroy_process_group()
+
+
+def test_sharded_gram_buffers_add_up_to_the_whole_problem():
+    """Every sum over the parameter index in the method is a sum over column slices and the centring is linear:
+    the all-reduced per-slice buffers equal the whole problem's centred Gram and G^T gbar (the fact that
+    qn_update_sharded rests on)."""
+    import numpy as np
+
+    sys.path.insert(0, ROOT)
+    import oracle
+    import workloads as W
+
+    world, port = 2, _free_port()
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_shard_rank_main, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    cfg = W.Config(21, 6003, 5, "f32", -1, 1, 0, 0.1, 1e-3, 1.0, 0.01)
+    theta, g = W.generate(cfg, "cpu")
+    gb = W.to_bits(g)
+    C = oracle.gram(gb)
+    g64 = oracle.storage_to_f64(gb)
+    gbar = g64.mean(0)
+    w = (g64 - gbar) @ gbar
+    whole = np.concatenate([C.reshape(-1), w])
+    assert np.array_equal(res[0], res[1])
+    scale = np.abs(C).max()
+    assert np.max(np.abs(res[0][: cfg.m ** 2] - whole[: cfg.m ** 2])) <= 1e-12 * scale
+    assert np.max(np.abs(res[0][cfg.m ** 2:] - whole[cfg.m ** 2:])) <= 1e-12 * max(np.abs(w).max(), scale)
