@@ -98,6 +98,15 @@ QN_API qn_status qn_update(qn_handle h, const void* theta, const void* g, double
                     void* theta_new, int32_t* j_out, double* sigma_out, void* cuda_stream);
 
 /*
+ * Cap on the number of modes: later steps on this handle keep at most j_cap of the modes that the lambda rule
+ * retains (the largest singular values); j_cap < 0 removes the cap (the default), j_cap = 0 gives the plain
+ * averaged-gradient step theta_bar - tau * g_bar (sentence after Eq. (4)).  Section 2 defines j through lambda
+ * only; Section 3 reports that the result depends strongly on how many singular values are considered, so the
+ * number can also be bounded directly.  sigma is still reported in full.  Host-side setting, no device work.
+ */
+QN_API qn_status qn_set_rank_cap(qn_handle h, int32_t j_cap);
+
+/*
  * The operator itself on an arbitrary vector: out = Hbar^{-1} z by Eq. (3)/(4),
  *   Hbar^{-1} z = z - sum_{k<=j} (u_k^T z) u_k + sum_{k<=j} (u_k^T z) sigma_k^{-1} y_k,
  * with u_k, y_k, sigma_k and the cut-off j built from (theta, g) exactly as in qn_update (qn_update is this

@@ -46,13 +46,14 @@ def lib() -> ctypes.CDLL:
         L.qno_eig.argtypes = [i32, vp, vp, vp]
         L.qno_cutoff.argtypes = [i32, vp, dbl, vp]
         L.qno_update.argtypes = [i64, i32, i32, vp, vp, dbl, dbl, vp, vp, i64, vp, vp, vp, vp, i32]
+        L.qno_update_capped.argtypes = [i64, i32, i32, vp, vp, dbl, dbl, i32, vp, vp, i64, vp, vp, vp, vp, i32]
         L.qno_apply_hinv.argtypes = [i64, i32, i32, vp, vp, dbl, vp, vp, vp, i32]
         L.qno_left_vectors.argtypes = [i64, i32, i32, vp, vp, dbl, vp, vp, vp, vp]
         L.qno_round_storage.argtypes = [i64, i32, vp, vp]
         L.qno_round_storage.restype = None
         L.qno_threads_used.argtypes = [i32]
-        for f in ("qno_gram", "qno_eig", "qno_cutoff", "qno_update", "qno_apply_hinv", "qno_left_vectors",
-                  "qno_threads_used"):
+        for f in ("qno_gram", "qno_eig", "qno_cutoff", "qno_update", "qno_update_capped", "qno_apply_hinv",
+                  "qno_left_vectors", "qno_threads_used"):
             getattr(L, f).restype = i32
         _lib = L
     return _lib
@@ -122,10 +123,11 @@ class UpdateResult:
 
 
 def update(theta: np.ndarray, g: np.ndarray, tau: float, lam: float, sample_idx: Optional[np.ndarray] = None,
-           nthreads: int = 0, want_theta: bool = True) -> UpdateResult:
+           nthreads: int = 0, want_theta: bool = True, j_cap: Optional[int] = None) -> UpdateResult:
     """Eq. (2): theta_new = thetabar - tau * Hinv gbar, in fp64.
 
-    With ``sample_idx`` (int64 column indices) only those entries of theta_new are evaluated."""
+    With ``sample_idx`` (int64 column indices) only those entries of theta_new are evaluated.  ``j_cap`` keeps at
+    most that many of the modes that the lambda rule retains (the largest ones)."""
     m, n, dt = _check_pair(theta, g)
     idx = None
     cnt = n
@@ -137,8 +139,9 @@ def update(theta: np.ndarray, g: np.ndarray, tau: float, lam: float, sample_idx:
     V = np.empty((m, m), dtype=np.float64)
     alpha = np.empty(m, dtype=np.float64)
     j = ctypes.c_int(0)
-    rc = lib().qno_update(n, m, dt, _ptr(theta), _ptr(g), float(tau), float(lam), _ptr(out), _ptr(idx), cnt,
-                          ctypes.byref(j), _ptr(sigma), _ptr(V), _ptr(alpha), nthreads)
+    rc = lib().qno_update_capped(n, m, dt, _ptr(theta), _ptr(g), float(tau), float(lam),
+                                 -1 if j_cap is None else int(j_cap), _ptr(out), _ptr(idx), cnt,
+                                 ctypes.byref(j), _ptr(sigma), _ptr(V), _ptr(alpha), nthreads)
     _raise(rc, "qno_update")
     return UpdateResult(out, j.value, sigma, V, alpha)
 

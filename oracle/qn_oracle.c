@@ -351,14 +351,17 @@ static inline double qno_hinv_column(int64_t n, int m, int dtype, const void* th
 }
 
 /* Shared front end: Gram, eigenpairs, cut-off, projections. */
-static int qno_front(int64_t n, int m, int dtype, const void* g, double lambda, const double* z, double* V,
+static int qno_front(int64_t n, int m, int dtype, const void* g, double lambda, int j_cap, const double* z, double* V,
                      double* sigma, int* j_out, double* gvnorm, double* alpha, int nthreads) {
     double C[QNO_MAX_M * QNO_MAX_M], mu[QNO_MAX_M];
     int rc = qno_gram(n, m, dtype, g, C, nthreads);
     if (rc) return rc;
     rc = qno_eig(m, C, V, mu);
     if (rc) return rc;
-    const int j = qno_cutoff(m, mu, lambda, sigma);
+    int j = qno_cutoff(m, mu, lambda, sigma);
+    /* optional cap on the number of modes kept (the parameter j of Section 2 set from outside; Section 3
+       stresses how much the result depends on it): the j_cap largest of those the lambda rule keeps */
+    if (j_cap >= 0 && j > j_cap) j = j_cap;
     *j_out = j;
     return qno_project(n, m, dtype, g, V, j, z, gvnorm, alpha, nthreads);
 }
@@ -372,13 +375,13 @@ static int qno_front(int64_t n, int m, int dtype, const void* g, double lambda, 
  *   sigma[m], V[m*m] (row-major, column k = v_k), alpha[m] (first j valid): optional outputs
  * Returns 0, or 1 bad argument, 2 out of memory, 3 Jacobi did not converge.
  */
-int qno_update(int64_t n, int m, int dtype, const void* theta, const void* g, double tau, double lambda,
-               double* theta_new, const int64_t* sample_idx, int64_t ns, int* j_out, double* sigma_out,
-               double* V_out, double* alpha_out, int nthreads) {
+int qno_update_capped(int64_t n, int m, int dtype, const void* theta, const void* g, double tau, double lambda,
+                      int j_cap, double* theta_new, const int64_t* sample_idx, int64_t ns, int* j_out,
+                      double* sigma_out, double* V_out, double* alpha_out, int nthreads) {
     if (n < 1 || m < 1 || m > QNO_MAX_M || !(lambda > 0.0)) return 1;
     double V[QNO_MAX_M * QNO_MAX_M], sigma[QNO_MAX_M], gvnorm[QNO_MAX_M], alpha[QNO_MAX_M];
     int j = 0;
-    int rc = qno_front(n, m, dtype, g, lambda, NULL, V, sigma, &j, gvnorm, alpha, nthreads);
+    int rc = qno_front(n, m, dtype, g, lambda, j_cap, NULL, V, sigma, &j, gvnorm, alpha, nthreads);
     if (rc) return rc;
     if (theta_new) {
         const int64_t cnt = sample_idx ? ns : n;
@@ -401,13 +404,21 @@ int qno_update(int64_t n, int m, int dtype, const void* theta, const void* g, do
     return 0;
 }
 
+/* The Server step with the lambda rule alone (no cap on j). */
+int qno_update(int64_t n, int m, int dtype, const void* theta, const void* g, double tau, double lambda,
+               double* theta_new, const int64_t* sample_idx, int64_t ns, int* j_out, double* sigma_out,
+               double* V_out, double* alpha_out, int nthreads) {
+    return qno_update_capped(n, m, dtype, theta, g, tau, lambda, -1, theta_new, sample_idx, ns, j_out, sigma_out, V_out,
+                             alpha_out, nthreads);
+}
+
 /* Eq. (3)/(4) applied to an arbitrary z in R^n (n doubles): out = Hinv z. */
 int qno_apply_hinv(int64_t n, int m, int dtype, const void* theta, const void* g, double lambda,
                    const double* z, double* out, int* j_out, int nthreads) {
     if (n < 1 || m < 1 || m > QNO_MAX_M || !(lambda > 0.0) || !z || !out) return 1;
     double V[QNO_MAX_M * QNO_MAX_M], sigma[QNO_MAX_M], gvnorm[QNO_MAX_M], alpha[QNO_MAX_M];
     int j = 0;
-    int rc = qno_front(n, m, dtype, g, lambda, z, V, sigma, &j, gvnorm, alpha, nthreads);
+    int rc = qno_front(n, m, dtype, g, lambda, -1, z, V, sigma, &j, gvnorm, alpha, nthreads);
     if (rc) return rc;
     for (int64_t i = 0; i < n; ++i)
         out[i] = qno_hinv_column(n, m, dtype, theta, g, V, j, sigma, gvnorm, alpha, z, i, NULL);
@@ -424,7 +435,7 @@ int qno_left_vectors(int64_t n, int m, int dtype, const void* theta, const void*
     if (n < 1 || m < 1 || m > QNO_MAX_M || !(lambda > 0.0)) return 1;
     double V[QNO_MAX_M * QNO_MAX_M], sigma[QNO_MAX_M], gvnorm[QNO_MAX_M], alpha[QNO_MAX_M];
     int j = 0;
-    int rc = qno_front(n, m, dtype, g, lambda, NULL, V, sigma, &j, gvnorm, alpha, 1);
+    int rc = qno_front(n, m, dtype, g, lambda, -1, NULL, V, sigma, &j, gvnorm, alpha, 1);
     if (rc) return rc;
     for (int64_t i = 0; i < n; ++i) {
         double gbar, tbar;

@@ -22,6 +22,7 @@ struct qn_ctx {
     unsigned int* ticket;         // device, zero between launches
     int* error_word;              // device, set by a kernel that gave up on a bounded wait
     double* rhs;                  // device, m doubles: g_k^T z of qn_apply_hinv
+    int32_t j_cap;                // < 0: none
 
     // asynchronous window
     void* win_theta;
@@ -147,6 +148,7 @@ qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, do
     }
     qn_solve_params p;
     memset(&p, 0, sizeof(p));
+    p.j_cap = h->j_cap;
     p.m = h->m;
     p.source = QN_SRC_PARTIALS;
     p.partials = h->partials;
@@ -211,6 +213,7 @@ extern "C" qn_status qn_create(int64_t n, int32_t m, qn_dtype dtype, qn_handle* 
     h->elem = dtype == QN_F32 ? 4 : 2;
     h->device = dev;
     h->last_sweeps = -1;
+    h->j_cap = -1;
     h->max_partials = qn_sm_count() * 4;
     bool ok = cudaMalloc(&h->partials, sizeof(double) * (size_t)h->max_partials * qn_partial_len(m)) == cudaSuccess;
     ok = ok && cudaMalloc(&h->coef, sizeof(qn_coef_block)) == cudaSuccess;
@@ -260,6 +263,12 @@ extern "C" qn_status qn_destroy(qn_handle h) {
     return QN_OK;
 }
 
+extern "C" qn_status qn_set_rank_cap(qn_handle h, int32_t j_cap) {
+    if (!h) return QN_ERR_INVALID;
+    h->j_cap = j_cap < 0 ? -1 : j_cap;
+    return QN_OK;
+}
+
 extern "C" qn_status qn_update(qn_handle h, const void* theta, const void* g, double tau, double lambda,
                                void* theta_new, int32_t* j_out, double* sigma_out, void* cuda_stream) {
     qn_status s = check_step_args(h, tau, lambda, theta_new);
@@ -294,6 +303,7 @@ extern "C" qn_status qn_update_from_gram(qn_handle h, const void* theta, const v
     begin_call(h, st);
     qn_solve_params p;
     memset(&p, 0, sizeof(p));
+    p.j_cap = h->j_cap;
     p.m = h->m;
     p.source = QN_SRC_SUMMED;
     p.raw_gram = const_cast<double*>(gram);  // read only in this mode
@@ -351,6 +361,7 @@ extern "C" qn_status qn_apply_hinv(qn_handle h, const void* theta, const void* g
     if (s == QN_OK) {
         qn_solve_params p;
         memset(&p, 0, sizeof(p));
+        p.j_cap = h->j_cap;
         p.m = h->m;
         p.source = QN_SRC_PARTIALS;
         p.partials = h->partials;
@@ -389,6 +400,7 @@ extern "C" qn_status qn_gram(qn_handle h, const void* g, double* gram_out, void*
     if (s == QN_OK) {
         qn_solve_params p;
         memset(&p, 0, sizeof(p));
+        p.j_cap = h->j_cap;
         p.m = h->m;
         p.source = QN_SRC_PARTIALS;
         p.partials = h->partials;
@@ -471,6 +483,7 @@ extern "C" qn_status qn_update_window(qn_handle h, double tau, double lambda, vo
     begin_call(h, st);
     qn_solve_params p;
     memset(&p, 0, sizeof(p));
+    p.j_cap = h->j_cap;
     p.m = h->m;
     p.source = QN_SRC_WINDOW;
     p.raw_gram = h->raw_gram;
@@ -510,6 +523,7 @@ extern "C" qn_status qn_rebuild(qn_handle h, void* cuda_stream) {
     if (s == QN_OK) {
         qn_solve_params p;
         memset(&p, 0, sizeof(p));
+        p.j_cap = h->j_cap;
         p.m = h->m;
         p.source = QN_SRC_PARTIALS;
         p.partials = h->partials;

@@ -58,6 +58,7 @@ struct qn_solve_params {
     double* gram_out;     // m*m + m doubles: centred C then w (may be NULL)
     int32_t gram_only;    // stop after writing gram_out
     double tau, lambda;
+    int32_t j_cap;        // < 0: no cap; else at most this many of the modes kept by the lambda rule
     const double* rhs_raw;  // NULL, or m doubles g_k^T z: the coefficients are then built for z instead of gbar
                             // (w = P rhs_raw) and with tau = -1, i.e. for out = z - G d + Theta d (Eq. (4))
     qn_coef_block* coef;

@@ -317,6 +317,7 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
         if (s1 > 0.0)
             for (int k = 0; k < m; ++k) j += (sm.sigma[k] >= prm.lambda * s1 && sm.sigma[k] > 0.0);
         if (j > m - 1) j = m - 1;
+        if (prm.j_cap >= 0 && j > prm.j_cap) j = prm.j_cap;  // the caller's cap on the number of modes
         sm.j = j;
     }
     asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");

@@ -392,6 +392,27 @@ def test_apply_hinv_is_the_identity_when_no_mode_is_kept(qn):
     assert j == 0 and status == 0 and torch.equal(out, z)
 
 
+@pytest.mark.parametrize("dtype,m,n", [("f32", 12, 30_000), ("bf16", 32, (1 << 22) + 8)])
+def test_rank_cap(qn, dtype, m, n):
+    """qn_set_rank_cap: cap 0 is the averaged-gradient step, a cap inside the retained modes matches the oracle with
+    the same cap, removing the cap restores the lambda rule."""
+    cfg = W.Config(45, n, m, dtype, -1, 1, 0, 0.1, 1e-3, 0.7, 0.02)
+    theta, g = W.generate(cfg, "cuda", gap_lam=cfg.lam, gap_scale=1.0)
+    tb, gb = W.to_bits(theta), W.to_bits(g)
+    free = oracle.update(tb, gb, cfg.tau, cfg.lam)
+    assert free.j >= 3
+    out = torch.empty(n, dtype=theta.dtype, device="cuda")
+    with qn.qn_create(n, m, theta.dtype) as h:
+        for cap in (0, 2, None):
+            qn.qn_set_rank_cap(h, cap)
+            j, sigma, status = qn.qn_update(h, theta, g, cfg.tau, cfg.lam, out)
+            ref = oracle.update(tb, gb, cfg.tau, cfg.lam, j_cap=cap)
+            assert status == 0 and j == ref.j == (free.j if cap is None else cap)
+            assert np.max(np.abs(np.array(sigma) - free.sigma)) <= 1e-5 * free.sigma[0]
+            got = oracle.storage_to_f64(W.to_bits(out))
+            assert np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL[dtype]
+
+
 # --------------------------------------------------------------------------- n-sharded step
 @pytest.mark.parametrize("dtype,m,n,shards", [("f32", 12, 40_008, 2), ("bf16", 8, 100_000, 3), ("f32", 32, (1 << 22) + 64, 2)])
 def test_sharded_step_matches_the_whole_problem(qn, dtype, m, n, shards):

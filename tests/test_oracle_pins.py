@@ -225,6 +225,37 @@ def test_p8_collapse_identity():
     np.testing.assert_allclose(r.theta_new, expect, rtol=0, atol=1e-11 * np.linalg.norm(expect))
 
 
+def test_p8_rank_cap():
+    """A cap on j keeps the largest of the modes that the lambda rule retains: cap 0 is the SGD step, a cap at or
+    above the rule's j changes nothing, and a cap in between equals the collapsed form built with numpy from
+    LAPACK's SVD truncated at the cap."""
+    rng = np.random.default_rng(18)
+    n, m, tau, lam = 48, 8, 0.3, 0.02
+    theta, g, _, _ = _rand_problem(rng, n, m, noise=0.02)
+    g = _as_f32_exact(g * np.geomspace(1, 0.1, n)[None, :])
+    t64, g64 = theta.astype(np.float64), g.astype(np.float64)
+    gbar, tbar = g64.mean(0), t64.mean(0)
+    G, Th = (g64 - gbar).T, (t64 - tbar).T
+    _, ss, Vt = np.linalg.svd(G, full_matrices=False)
+    free = oracle.update(theta, g, tau, lam)
+    assert free.j >= 4
+    r0 = oracle.update(theta, g, tau, lam, j_cap=0)
+    assert r0.j == 0
+    np.testing.assert_allclose(r0.theta_new, tbar - tau * gbar, rtol=0, atol=1e-14 * np.linalg.norm(tbar))
+    for cap in (free.j, free.j + 1, m):
+        r = oracle.update(theta, g, tau, lam, j_cap=cap)
+        assert r.j == free.j and np.array_equal(r.theta_new, free.theta_new)
+    for cap in (1, 3):
+        Vj = Vt[:cap].T
+        d = Vj @ ((Vj.T @ (G.T @ gbar)) / ss[:cap] ** 2)
+        expect = tbar - tau * (gbar - G @ d + Th @ d)
+        r = oracle.update(theta, g, tau, lam, j_cap=cap)
+        assert r.j == cap
+        np.testing.assert_allclose(r.theta_new, expect, rtol=0, atol=1e-11 * np.linalg.norm(expect))
+        np.testing.assert_array_equal(r.sigma, free.sigma)  # sigma is reported in full whatever the cap
+        assert np.linalg.norm(r.theta_new - free.theta_new) > 1e-6 * np.linalg.norm(free.theta_new)
+
+
 # ---------------------------------------------------------------- P9: symmetries
 def test_p9_symmetries():
     rng = np.random.default_rng(9)
