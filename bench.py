@@ -315,7 +315,8 @@ def main():
     dominant = max(per_kernel, key=lambda k: per_kernel[k][0] * per_kernel[k][1])
     dom_ms = per_kernel[dominant][0]
     achieved = bytes_per[dominant] / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 and bytes_per[dominant] else 0.0
-    ratio = MEASURED_TRAFFIC_RATIO.get((dominant, cfg.dtype, "tc" if cfg.m > 8 else "direct"))
+    path = "tc" if (cfg.m > 8 and cfg.n >= (1 << 22)) else "direct" if cfg.m <= 8 else "alu"
+    ratio = MEASURED_TRAFFIC_RATIO.get((dominant, cfg.dtype, path))
     roofline = {
         "bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
         "frac": achieved / peak if peak else None, "peak_kind": "of " + peak_kind,
