@@ -107,6 +107,21 @@ QN_API qn_status qn_update(qn_handle h, const void* theta, const void* g, double
 QN_API qn_status qn_set_rank_cap(qn_handle h, int32_t j_cap);
 
 /*
+ * Learning-rate cap (Section 3, last paragraph: the optimal rate is 1 / sigma_max of the Hessian, and the method
+ * approximates sigma_max itself, so the rate can be bounded by it at every update).  The operator is built from
+ * the pairs Hbar y_k = sigma_k u_k with y_k = Theta v_k (Eq. (1), text before Eq. (3)); the Hessian's largest
+ * singular value as the method sees it is max_{k<=j} sigma_k / ||y_k||_2, and with the cap on, qn_update and
+ * qn_update_host use tau_eff = min(tau, 1 / that) when tau > 0.  ||y_k||^2 = v_k^T (Theta^T Theta) v_k needs the
+ * Gram of theta: one more streaming pass (m*n elements read, a fourth kernel launch).  The asynchronous window,
+ * qn_update_from_gram and qn_apply_hinv ignore the setting.
+ *   on           0 = off (default), else on; the first switch-on allocates the pass's partial sums on the device
+ * qn_last_tau returns the rate used by the most recent step whose results were fetched to the host
+ * (j_out or sigma_out non-NULL, or qn_status_sync).
+ */
+QN_API qn_status qn_set_tau_cap(qn_handle h, int32_t on);
+QN_API double qn_last_tau(qn_handle h);
+
+/*
  * The operator itself on an arbitrary vector: out = Hbar^{-1} z by Eq. (3)/(4),
  *   Hbar^{-1} z = z - sum_{k<=j} (u_k^T z) u_k + sum_{k<=j} (u_k^T z) sigma_k^{-1} y_k,
  * with u_k, y_k, sigma_k and the cut-off j built from (theta, g) exactly as in qn_update (qn_update is this

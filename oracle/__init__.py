@@ -46,7 +46,7 @@ def lib() -> ctypes.CDLL:
         L.qno_eig.argtypes = [i32, vp, vp, vp]
         L.qno_cutoff.argtypes = [i32, vp, dbl, vp]
         L.qno_update.argtypes = [i64, i32, i32, vp, vp, dbl, dbl, vp, vp, i64, vp, vp, vp, vp, i32]
-        L.qno_update_capped.argtypes = [i64, i32, i32, vp, vp, dbl, dbl, i32, vp, vp, i64, vp, vp, vp, vp, i32]
+        L.qno_update_capped.argtypes = [i64, i32, i32, vp, vp, dbl, dbl, i32, i32, vp, vp, i64, vp, vp, vp, vp, vp, i32]
         L.qno_apply_hinv.argtypes = [i64, i32, i32, vp, vp, dbl, vp, vp, vp, i32]
         L.qno_left_vectors.argtypes = [i64, i32, i32, vp, vp, dbl, vp, vp, vp, vp]
         L.qno_round_storage.argtypes = [i64, i32, vp, vp]
@@ -116,18 +116,21 @@ def cutoff(mu: np.ndarray, lam: float):
 
 
 class UpdateResult:
-    __slots__ = ("theta_new", "j", "sigma", "V", "alpha")
+    __slots__ = ("theta_new", "j", "sigma", "V", "alpha", "tau_eff")
 
-    def __init__(self, theta_new, j, sigma, V, alpha):
-        self.theta_new, self.j, self.sigma, self.V, self.alpha = theta_new, j, sigma, V, alpha
+    def __init__(self, theta_new, j, sigma, V, alpha, tau_eff=None):
+        self.theta_new, self.j, self.sigma, self.V, self.alpha, self.tau_eff = theta_new, j, sigma, V, alpha, tau_eff
 
 
 def update(theta: np.ndarray, g: np.ndarray, tau: float, lam: float, sample_idx: Optional[np.ndarray] = None,
-           nthreads: int = 0, want_theta: bool = True, j_cap: Optional[int] = None) -> UpdateResult:
+           nthreads: int = 0, want_theta: bool = True, j_cap: Optional[int] = None,
+           tau_cap: bool = False) -> UpdateResult:
     """Eq. (2): theta_new = thetabar - tau * Hinv gbar, in fp64.
 
     With ``sample_idx`` (int64 column indices) only those entries of theta_new are evaluated.  ``j_cap`` keeps at
-    most that many of the modes that the lambda rule retains (the largest ones)."""
+    most that many of the modes that the lambda rule retains (the largest ones).  ``tau_cap`` bounds tau by
+    1 / max_k (sigma_k / ||Theta v_k||), the method's own estimate of the Hessian's largest singular value
+    (Section 3, last paragraph); the rate used is returned as ``tau_eff``."""
     m, n, dt = _check_pair(theta, g)
     idx = None
     cnt = n
@@ -139,11 +142,12 @@ def update(theta: np.ndarray, g: np.ndarray, tau: float, lam: float, sample_idx:
     V = np.empty((m, m), dtype=np.float64)
     alpha = np.empty(m, dtype=np.float64)
     j = ctypes.c_int(0)
+    tau_eff = ctypes.c_double(0.0)
     rc = lib().qno_update_capped(n, m, dt, _ptr(theta), _ptr(g), float(tau), float(lam),
-                                 -1 if j_cap is None else int(j_cap), _ptr(out), _ptr(idx), cnt,
-                                 ctypes.byref(j), _ptr(sigma), _ptr(V), _ptr(alpha), nthreads)
+                                 -1 if j_cap is None else int(j_cap), 1 if tau_cap else 0, _ptr(out), _ptr(idx), cnt,
+                                 ctypes.byref(j), _ptr(sigma), _ptr(V), _ptr(alpha), ctypes.byref(tau_eff), nthreads)
     _raise(rc, "qno_update")
-    return UpdateResult(out, j.value, sigma, V, alpha)
+    return UpdateResult(out, j.value, sigma, V, alpha, tau_eff.value)
 
 
 def apply_hinv(theta: np.ndarray, g: np.ndarray, lam: float, z: np.ndarray, nthreads: int = 0):

@@ -375,14 +375,31 @@ static int qno_front(int64_t n, int m, int dtype, const void* g, double lambda, 
  *   sigma[m], V[m*m] (row-major, column k = v_k), alpha[m] (first j valid): optional outputs
  * Returns 0, or 1 bad argument, 2 out of memory, 3 Jacobi did not converge.
  */
+/*
+ * tau_cap != 0: the learning rate is bounded by the reciprocal of the largest singular value of the Hessian as
+ * the method itself sees it (last paragraph of Section 3: tau_opt = 1 / sigma_max, "we directly approximate
+ * sigma_max").  The operator is built from the pairs Hbar y_k = sigma_k u_k (Eq. (1) and the text before
+ * Eq. (3)), so the estimate is max_{k<=j} ||Hbar y_k|| / ||y_k|| = max_k sigma_k / ||Theta v_k||_2, and
+ * tau_eff = min(tau, 1 / that) for tau > 0.  tau_eff_out (may be NULL) receives the rate that was used.
+ */
 int qno_update_capped(int64_t n, int m, int dtype, const void* theta, const void* g, double tau, double lambda,
-                      int j_cap, double* theta_new, const int64_t* sample_idx, int64_t ns, int* j_out,
-                      double* sigma_out, double* V_out, double* alpha_out, int nthreads) {
+                      int j_cap, int tau_cap, double* theta_new, const int64_t* sample_idx, int64_t ns, int* j_out,
+                      double* sigma_out, double* V_out, double* alpha_out, double* tau_eff_out, int nthreads) {
     if (n < 1 || m < 1 || m > QNO_MAX_M || !(lambda > 0.0)) return 1;
     double V[QNO_MAX_M * QNO_MAX_M], sigma[QNO_MAX_M], gvnorm[QNO_MAX_M], alpha[QNO_MAX_M];
     int j = 0;
     int rc = qno_front(n, m, dtype, g, lambda, j_cap, NULL, V, sigma, &j, gvnorm, alpha, nthreads);
     if (rc) return rc;
+    if (tau_cap && j > 0 && tau > 0.0) {
+        double ynorm[QNO_MAX_M], unused[QNO_MAX_M];
+        rc = qno_project(n, m, dtype, theta, V, j, NULL, ynorm, unused, nthreads); /* ||Theta v_k||_2 */
+        if (rc) return rc;
+        double smax = 0.0;
+        for (int k = 0; k < j; ++k)
+            if (ynorm[k] > 0.0 && sigma[k] / ynorm[k] > smax) smax = sigma[k] / ynorm[k];
+        if (smax > 0.0 && 1.0 / smax < tau) tau = 1.0 / smax;
+    }
+    if (tau_eff_out) *tau_eff_out = tau;
     if (theta_new) {
         const int64_t cnt = sample_idx ? ns : n;
         const int nt = qno_threads(nthreads);
@@ -408,8 +425,8 @@ int qno_update_capped(int64_t n, int m, int dtype, const void* theta, const void
 int qno_update(int64_t n, int m, int dtype, const void* theta, const void* g, double tau, double lambda,
                double* theta_new, const int64_t* sample_idx, int64_t ns, int* j_out, double* sigma_out,
                double* V_out, double* alpha_out, int nthreads) {
-    return qno_update_capped(n, m, dtype, theta, g, tau, lambda, -1, theta_new, sample_idx, ns, j_out, sigma_out, V_out,
-                             alpha_out, nthreads);
+    return qno_update_capped(n, m, dtype, theta, g, tau, lambda, -1, 0, theta_new, sample_idx, ns, j_out, sigma_out,
+                             V_out, alpha_out, NULL, nthreads);
 }
 
 /* Eq. (3)/(4) applied to an arbitrary z in R^n (n doubles): out = Hinv z. */

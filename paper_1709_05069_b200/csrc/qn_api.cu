@@ -23,6 +23,9 @@ struct qn_ctx {
     int* error_word;              // device, set by a kernel that gave up on a bounded wait
     double* rhs;                  // device, m doubles: g_k^T z of qn_apply_hinv
     int32_t j_cap;                // < 0: none
+    int32_t tau_cap;              // learning-rate cap on/off (qn_update and qn_update_host)
+    double* partials_theta;       // device, as `partials`, allocated when the cap is first switched on
+    double last_tau;              // learning rate of the most recent step whose results were fetched
 
     // asynchronous window
     void* win_theta;
@@ -122,6 +125,7 @@ qn_status fetch_result(qn_handle h, cudaStream_t st, int32_t* j_out, double* sig
     if (j_out) *j_out = h->host_result->j;
     if (sigma_out) memcpy(sigma_out, h->host_result->sigma, sizeof(double) * h->m);
     h->last_sweeps = h->host_result->sweeps;
+    h->last_tau = h->host_result->tau_eff;
     return static_cast<qn_status>(h->host_result->status);
 }
 
@@ -146,9 +150,20 @@ qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, do
                            &h->last_launches, h->error_word) != cudaSuccess)
             return QN_ERR_CUDA;
     }
+    int np_theta = 0;
+    if (h->tau_cap && h->partials_theta) {
+        // the learning-rate cap needs ||Theta v_k||: one more Gram pass, over theta
+        KernelTimer t(h, st, QN_TIME_GRAM);
+        if (qn_launch_gram(h->dtype, theta, h->n, h->m, false, h->partials_theta, &np_theta, h->max_partials, st,
+                           &h->last_launches, h->error_word) != cudaSuccess)
+            return QN_ERR_CUDA;
+    }
     qn_solve_params p;
     memset(&p, 0, sizeof(p));
     p.j_cap = h->j_cap;
+    p.tau_cap = h->tau_cap && h->partials_theta;
+    p.partials_theta = h->partials_theta;
+    p.num_partials_theta = np_theta;
     p.m = h->m;
     p.source = QN_SRC_PARTIALS;
     p.partials = h->partials;
@@ -246,6 +261,7 @@ extern "C" qn_status qn_destroy(qn_handle h) {
     cudaFree(h->raw_gram);
     cudaFree(h->ticket);
     cudaFree(h->rhs);
+    cudaFree(h->partials_theta);
     cudaFree(h->error_word);
     cudaFree(h->win_theta);
     cudaFree(h->win_g);
@@ -262,6 +278,24 @@ extern "C" qn_status qn_destroy(qn_handle h) {
     delete h;
     return QN_OK;
 }
+
+extern "C" qn_status qn_set_tau_cap(qn_handle h, int32_t on) {
+    if (!h) return QN_ERR_INVALID;
+    if (on && !h->partials_theta) {
+        DeviceGuard guard(h->device);
+        if (!guard.ok) return QN_ERR_CUDA;
+        if (cudaMalloc(&h->partials_theta, sizeof(double) * (size_t)h->max_partials * qn_partial_len(h->m)) !=
+            cudaSuccess) {
+            cudaGetLastError();
+            h->partials_theta = nullptr;
+            return QN_ERR_ALLOC;
+        }
+    }
+    h->tau_cap = on ? 1 : 0;
+    return QN_OK;
+}
+
+extern "C" double qn_last_tau(qn_handle h) { return h ? h->last_tau : 0.0; }
 
 extern "C" qn_status qn_set_rank_cap(qn_handle h, int32_t j_cap) {
     if (!h) return QN_ERR_INVALID;

@@ -243,7 +243,8 @@ __global__ void __launch_bounds__(kGsThreads, 1)
 gram_stream_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ partials, int* __restrict__ error_word) {
     constexpr int kCols = Storage<T>::kVec;
     constexpr int kTileCols = kGsSeg / (int)sizeof(T);
-    constexpr int kFlushIters = kFlushCols / kCols;
+    // each half of a packed accumulator sums every other column: kFlushCols columns per half between flushes
+    constexpr int kFlushIters = 2 * kFlushCols / kCols;
     extern __shared__ unsigned char smem_raw[];
     GsSmem& sm = *reinterpret_cast<GsSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -314,7 +315,8 @@ gram_stream_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict
                 for (int k = 1; k < kDirectM; ++k) sum = gs_add2(sum, x[k]);
                 const uint64_t r = gs_mul2(sum, inv_m2);
 #pragma unroll
-                for (int k = 0; k < kDirectM; ++k) x[k] = k < m ? gs_sub2(x[k], r) : 0ull;  // padding rows stay zero
+                // padding rows (k >= m) read as zero and become -r here: they only reach sums that are never output
+                for (int k = 0; k < kDirectM; ++k) x[k] = gs_sub2(x[k], r);
 #pragma unroll
                 for (int k = 0, idx = 0; k < kDirectM; ++k) {
 #pragma unroll
@@ -596,6 +598,11 @@ static bool tc_allowed() {
     const char* v = getenv("QN_GRAM_PATH");
     return !(v && v[0] == 'a');
 }
+// QN_GRAM_PATH=stream sends bf16 storage to the bulk-copy direct kernel as well (A/B measurements)
+static bool stream_forced() {
+    const char* v = getenv("QN_GRAM_PATH");
+    return v && v[0] == 's';
+}
 
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
                            int* num_partials, int max_partials, cudaStream_t st, int* launches, int* error_word) {
@@ -603,14 +610,17 @@ cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool
     const int64_t elem = dtype == QN_F32 ? 4 : 2;
     if (!raw && tc_allowed() && qn_gram_tc_applicable(dtype, g, n, m)) {
         e = qn_launch_gram_tc(dtype, g, n, m, partials, num_partials, max_partials, error_word, st);
-    } else if (!raw && tc_allowed() && dtype == QN_F32 && m <= qn::kDirectM && n >= QN_PRECISE_BELOW &&
-               reinterpret_cast<uintptr_t>(g) % 16 == 0 && (n * elem) % 16 == 0) {
-        // Bulk-copy variant of the direct kernel (QN_GRAM_PATH=alu keeps the register-fed one, for A/B runs).
-        // Measured at m = 8: fp32 storage 6.0 TB/s against 5.3 TB/s register-fed; bf16 storage 4.0 against 4.3
-        // (there both are bound by the instructions per element, and seven warps hide latency worse than eight
-        // with register prefetch), so bf16 storage stays on the register-fed kernel.
-        e = qn::launch_gram_stream(static_cast<const float*>(g), n, m, partials, num_partials, max_partials,
-                                   error_word, st);
+    } else if (!raw && tc_allowed() && (dtype == QN_F32 || m == qn::kDirectM || stream_forced()) && m <= qn::kDirectM &&
+               n >= QN_PRECISE_BELOW && reinterpret_cast<uintptr_t>(g) % 16 == 0 && (n * elem) % 16 == 0) {
+        // Bulk-copy variant of the direct kernel (QN_GRAM_PATH=alu keeps the register-fed one, QN_GRAM_PATH=stream
+        // forces this one, for A/B runs).  Measured: fp32 storage 6.4 TB/s at m = 8 and 4.9 at m = 5 against 5.3 and
+        // 3.8 register-fed; bf16 storage 4.5 against 4.3 at m = 8 but 2.3 against 2.4 at m = 4 (with bf16 both are
+        // bound by the instructions per element, which do not shrink with m because all eight rows are always
+        // computed), so bf16 storage comes here only with eight Workers.
+        e = dtype == QN_F32 ? qn::launch_gram_stream(static_cast<const float*>(g), n, m, partials, num_partials,
+                                                     max_partials, error_word, st)
+                            : qn::launch_gram_stream(static_cast<const __nv_bfloat16*>(g), n, m, partials,
+                                                     num_partials, max_partials, error_word, st);
     } else {
         e = dtype == QN_F32
                 ? qn::launch_gram_t(static_cast<const float*>(g), n, m, raw, partials, num_partials, max_partials, st)

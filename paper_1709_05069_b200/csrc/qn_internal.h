@@ -29,6 +29,7 @@ struct qn_result_block {
     int32_t sweeps;
     int32_t pad;
     double sigma[QN_MAX_M];
+    double tau_eff;  // the learning rate the step used (tau, or less under the learning-rate cap)
 };
 
 // Coefficients consumed by the combine kernel:
@@ -59,6 +60,9 @@ struct qn_solve_params {
     int32_t gram_only;    // stop after writing gram_out
     double tau, lambda;
     int32_t j_cap;        // < 0: no cap; else at most this many of the modes kept by the lambda rule
+    int32_t tau_cap;      // != 0 with partials_theta: tau <- min(tau, 1 / max_k sigma_k / ||Theta v_k||)
+    const double* partials_theta;  // Gram partials of theta (same layout as `partials`), or NULL
+    int32_t num_partials_theta;
     const double* rhs_raw;  // NULL, or m doubles g_k^T z: the coefficients are then built for z instead of gbar
                             // (w = P rhs_raw) and with tau = -1, i.e. for out = z - G d + Theta d (Eq. (4))
     qn_coef_block* coef;

@@ -22,6 +22,7 @@ constexpr int kMaxSweeps = 30;
 struct SolveSmem {
     double A[QN_MAX_M * kLd];
     double V[QN_MAX_M * kLd];  // also scratch for the partial sums before the Jacobi phase
+    double B[QN_MAX_M * kLd];  // reference-shifted Gram of theta (learning-rate cap only)
     double w[QN_MAX_M];
     double rowsum[QN_MAX_M];
     double mu[QN_MAX_M];
@@ -36,6 +37,7 @@ struct SolveSmem {
     int flag_rotated;
     int flag_timeout;
     int j;
+    double tau_eff;
 };
 
 __device__ __forceinline__ double block_sum(double x, double* red) {
@@ -107,6 +109,26 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
         __syncthreads();
         if (prm.raw_gram)
             for (int e = tid; e < m * m; e += nthr) prm.raw_gram[e] = sm.A[(e / m) * kLd + (e % m)];
+        if (prm.tau_cap && prm.partials_theta) {
+            // the same fixed-order sum for the Gram of theta; it stays reference-shifted: it is only ever applied
+            // to retained v_k, which are orthogonal to the vector of ones, so the centring would change nothing
+            for (int e = tid; e < tri_len; e += nthr) {
+                double s0 = 0, s1 = 0;
+                int p = 0;
+                for (; p + 1 < prm.num_partials_theta; p += 2) {
+                    s0 += prm.partials_theta[(int64_t)(p + 0) * E + e];
+                    s1 += prm.partials_theta[(int64_t)(p + 1) * E + e];
+                }
+                if (p < prm.num_partials_theta) s0 += prm.partials_theta[(int64_t)p * E + e];
+                packed[e] = s0 + s1;
+            }
+            __syncthreads();
+            for (int e = tid; e < m * m; e += nthr) {
+                const int k = e / m, l = e % m;
+                sm.B[k * kLd + l] = packed[k <= l ? qn_tri_index(m, k, l) : qn_tri_index(m, l, k)];
+            }
+            __syncthreads();
+        }
     } else {
         // QN_SRC_WINDOW: the raw Gram (w follows from it in the centring below); QN_SRC_SUMMED: a centred Gram
         // followed by w, e.g. the sum over column shards of what qn_gram wrote (the centring below leaves an
@@ -176,6 +198,7 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
             prm.result->j = 0;
             prm.result->status = sm.flag_timeout ? QN_ERR_DEVICE_TIMEOUT : QN_ERR_NONFINITE;
             prm.result->sweeps = 0;
+            prm.result->tau_eff = prm.tau;
         }
         return;
     }
@@ -322,6 +345,33 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
     }
     asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
     const int j = sm.j;
+    // Learning-rate cap (Section 3, last paragraph: tau_opt = 1 / sigma_max of the Hessian).  The operator is built
+    // from Hbar y_k = sigma_k u_k, so the Hessian's largest singular value as the method sees it is
+    // max_k sigma_k / ||y_k||, with ||y_k||^2 = v_k^T (Theta^T Theta) v_k.
+    double tau_use = prm.tau;
+    if (prm.tau_cap && prm.partials_theta && prm.source == QN_SRC_PARTIALS && j > 0 && prm.tau > 0.0) {
+        for (int e = tid; e < j * m; e += jthreads) {  // A is free from here on: scratch for the j x m products
+            const int k = e / m, a = e % m, col = sm.order[k];
+            double bv = 0.0;
+            for (int b = 0; b < m; ++b) bv += sm.B[a * kLd + b] * sm.V[b * kLd + col];
+            sm.A[k * kLd + a] = sm.V[a * kLd + col] * bv;
+        }
+        asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
+        if (tid < j) {
+            double y2 = 0.0;
+            for (int a = 0; a < m; ++a) y2 += sm.A[tid * kLd + a];
+            sm.d[tid] = y2 > 0.0 ? sm.sigma[tid] / sqrt(y2) : 0.0;
+        }
+        asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
+        if (tid == 0) {
+            double smax = 0.0;
+            for (int k = 0; k < j; ++k) smax = fmax(smax, sm.d[k]);
+            sm.tau_eff = (smax > 0.0 && 1.0 / smax < prm.tau) ? 1.0 / smax : prm.tau;
+        }
+        asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
+        tau_use = sm.tau_eff;
+        asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");  // d is rewritten below
+    }
     if (tid < j) {
         const int col = sm.order[tid];
         double dot = 0.0;
@@ -338,13 +388,14 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
     if (tid < QN_MAX_M) {
         double s = 0.0;
         for (int k = 0; k < m; ++k) s += sm.d[k];
-        prm.coef->c[tid] = tid < m ? (float)(prm.tau * (sm.d[tid] - s * inv_m)) : 0.f;
+        prm.coef->c[tid] = tid < m ? (float)(tau_use * (sm.d[tid] - s * inv_m)) : 0.f;
         prm.result->sigma[tid] = tid < m ? sm.sigma[tid] : 0.0;
     }
     if (tid == 0) {
-        prm.coef->tau = (float)prm.tau;
+        prm.coef->tau = (float)tau_use;
         prm.coef->inv_m = (float)inv_m;
         prm.coef->m = m;
+        prm.result->tau_eff = tau_use;
         prm.result->j = j;
         prm.result->status = sm.flag_timeout ? QN_ERR_DEVICE_TIMEOUT : converged ? QN_OK : QN_ERR_NOT_CONVERGED;
         prm.result->sweeps = sweeps;

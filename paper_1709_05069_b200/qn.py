@@ -22,7 +22,7 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libqn.so")
 _lib: Optional[ctypes.CDLL] = None
 
 EXPORTS = (
-    "qn_strerror", "qn_create", "qn_destroy", "qn_update", "qn_gram", "qn_update_from_gram", "qn_apply_hinv", "qn_set_rank_cap", "qn_push", "qn_update_window", "qn_rebuild",
+    "qn_strerror", "qn_create", "qn_destroy", "qn_update", "qn_gram", "qn_update_from_gram", "qn_apply_hinv", "qn_set_rank_cap", "qn_set_tau_cap", "qn_last_tau", "qn_push", "qn_update_window", "qn_rebuild",
     "qn_window_alloc", "qn_window_theta", "qn_window_g", "qn_window_mark_full", "qn_update_host", "qn_status_sync",
     "qn_last_launches", "qn_total_launches", "qn_last_sweeps", "qn_timing_begin", "qn_timing_end",
     "qn_gram_static",
@@ -50,6 +50,8 @@ def lib() -> ctypes.CDLL:
         L.qn_destroy.argtypes, L.qn_destroy.restype = [vp], i32
         L.qn_update.argtypes, L.qn_update.restype = [vp, vp, vp, dbl, dbl, vp, vp, vp, vp], i32
         L.qn_gram.argtypes, L.qn_gram.restype = [vp, vp, vp, vp], i32
+        L.qn_set_tau_cap.argtypes, L.qn_set_tau_cap.restype = [vp, i32], i32
+        L.qn_last_tau.argtypes, L.qn_last_tau.restype = [vp], dbl
         L.qn_set_rank_cap.argtypes, L.qn_set_rank_cap.restype = [vp, i32], i32
         L.qn_apply_hinv.argtypes, L.qn_apply_hinv.restype = [vp, vp, vp, dbl, vp, vp, vp, vp, vp], i32
         L.qn_update_from_gram.argtypes, L.qn_update_from_gram.restype = [vp, vp, vp, vp, dbl, dbl, vp, vp, vp, vp], i32
@@ -187,6 +189,17 @@ def qn_gram(h: Handle, g: torch.Tensor, gram_out: torch.Tensor, stream=None) -> 
 def qn_set_rank_cap(h: Handle, j_cap: Optional[int]) -> None:
     """Keep at most ``j_cap`` modes in later steps on this handle (``None`` or a negative value: no cap)."""
     _check(lib().qn_set_rank_cap(h.ptr, -1 if j_cap is None else int(j_cap)), "qn_set_rank_cap")
+
+
+def qn_set_tau_cap(h: Handle, on: bool) -> None:
+    """Bound tau by the reciprocal of the method's estimate of the Hessian's largest singular value in later
+    ``qn_update`` / ``qn_update_host`` calls on this handle (one more pass, over theta)."""
+    _check(lib().qn_set_tau_cap(h.ptr, 1 if on else 0), "qn_set_tau_cap")
+
+
+def qn_last_tau(h: Handle) -> float:
+    """Learning rate used by the most recent step whose results were fetched to the host."""
+    return float(lib().qn_last_tau(h.ptr))
 
 
 def qn_apply_hinv(h: Handle, theta: torch.Tensor, g: torch.Tensor, lam: float, z: torch.Tensor, out: torch.Tensor,

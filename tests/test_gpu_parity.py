@@ -413,6 +413,34 @@ def test_rank_cap(qn, dtype, m, n):
             assert np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL[dtype]
 
 
+@pytest.mark.parametrize("dtype,m,n", [("f32", 8, 50_000), ("f32", 24, 20_000), ("bf16", 16, (1 << 22) + 8)])
+def test_learning_rate_cap(qn, dtype, m, n):
+    """qn_set_tau_cap: with a tau far above the bound the step uses 1 / max_k sigma_k / ||Theta v_k||, with a tau
+    below it nothing changes; both against the oracle's own evaluation of the bound."""
+    cfg = W.Config(46, n, m, dtype, -1, 1, 0, 0.1, 1e-3, 1.0, 0.02)
+    theta, g = W.generate(cfg, "cuda", gap_lam=cfg.lam, gap_scale=1.0)
+    tb, gb = W.to_bits(theta), W.to_bits(g)
+    big = oracle.update(tb, gb, 1e3, cfg.lam, tau_cap=True)
+    assert big.tau_eff < 1e3
+    out = torch.empty(n, dtype=theta.dtype, device="cuda")
+    with qn.qn_create(n, m, theta.dtype) as h:
+        qn.qn_set_tau_cap(h, True)
+        j, sigma, status = qn.qn_update(h, theta, g, 1e3, cfg.lam, out)
+        assert status == 0 and j == big.j and h.last_launches == 4
+        assert abs(qn.qn_last_tau(h) - big.tau_eff) <= 1e-5 * big.tau_eff
+        got = oracle.storage_to_f64(W.to_bits(out))
+        assert np.linalg.norm(got - big.theta_new) / np.linalg.norm(big.theta_new) <= TOL[dtype]
+        small = 0.1 * big.tau_eff
+        j, sigma, status = qn.qn_update(h, theta, g, small, cfg.lam, out)
+        assert qn.qn_last_tau(h) == small
+        ref = oracle.update(tb, gb, small, cfg.lam)
+        got = oracle.storage_to_f64(W.to_bits(out))
+        assert np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL[dtype]
+        qn.qn_set_tau_cap(h, False)
+        j, sigma, status = qn.qn_update(h, theta, g, 1e3, cfg.lam, out)
+        assert qn.qn_last_tau(h) == 1e3 and h.last_launches == 3
+
+
 # --------------------------------------------------------------------------- n-sharded step
 @pytest.mark.parametrize("dtype,m,n,shards", [("f32", 12, 40_008, 2), ("bf16", 8, 100_000, 3), ("f32", 32, (1 << 22) + 64, 2)])
 def test_sharded_step_matches_the_whole_problem(qn, dtype, m, n, shards):

@@ -256,6 +256,44 @@ def test_p8_rank_cap():
         assert np.linalg.norm(r.theta_new - free.theta_new) > 1e-6 * np.linalg.norm(free.theta_new)
 
 
+def test_p8_learning_rate_cap():
+    """tau is bounded by 1 / max_k sigma_k / ||Theta v_k||.  For noise-free gradients of a quadratic, G = A Theta
+    and sigma_k u_k = A y_k, so the estimate is a quotient ||A y|| / ||y||: it lies between the extreme singular
+    values of A, equals a for A = a I, and matches the same quantity built with numpy from LAPACK's SVD."""
+    rng = np.random.default_rng(28)
+    n, m, lam = 5, 9, 1e-6
+    for kind in ("scaled identity", "spd"):
+        if kind == "scaled identity":
+            A = 4.0 * np.eye(n)
+        else:
+            Q, _ = np.linalg.qr(rng.standard_normal((n, n)))
+            A = (Q * np.array([0.5, 1.0, 2.0, 3.0, 8.0])) @ Q.T
+            A = np.round(A * 1024) / 1024
+            A = (A + A.T) / 2
+        b = np.round(rng.standard_normal(n) * 64) / 64
+        theta = (np.round(rng.standard_normal((m, n)) * 64) / 64).astype(np.float32)
+        g = (theta.astype(np.float64) @ A.T - b).astype(np.float32)
+        assert np.array_equal(g.astype(np.float64), theta.astype(np.float64) @ A.T - b)  # exactly representable
+        t64, g64 = theta.astype(np.float64), g.astype(np.float64)
+        G, Th = (g64 - g64.mean(0)).T, (t64 - t64.mean(0)).T
+        _, ss, Vt = np.linalg.svd(G, full_matrices=False)
+        r_free = oracle.update(theta, g, 10.0, lam)
+        jj = r_free.j
+        est = max(ss[k] / np.linalg.norm(Th @ Vt[k]) for k in range(jj))
+        sv = np.linalg.svd(A, compute_uv=False)
+        assert sv[-1] * (1 - 1e-9) <= est <= sv[0] * (1 + 1e-9)
+        if kind == "scaled identity":
+            assert abs(est - 4.0) <= 1e-10
+        r = oracle.update(theta, g, 10.0, lam, tau_cap=True)   # 10 is far above 1 / est: capped
+        assert abs(r.tau_eff - 1.0 / est) <= 1e-9 / est
+        expect = t64.mean(0) + (r.tau_eff / 10.0) * (r_free.theta_new - t64.mean(0))  # the step scales with tau
+        np.testing.assert_allclose(r.theta_new, expect, rtol=0, atol=1e-10 * np.linalg.norm(expect))
+        small = 0.01 / est
+        r = oracle.update(theta, g, small, lam, tau_cap=True)  # below the bound: untouched
+        assert r.tau_eff == small
+        assert np.array_equal(r.theta_new, oracle.update(theta, g, small, lam).theta_new)
+
+
 # ---------------------------------------------------------------- P9: symmetries
 def test_p9_symmetries():
     rng = np.random.default_rng(9)
