@@ -142,25 +142,44 @@ __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
     return r;
 }
 
-// pair p of a 16-byte vector as two floats
+// One work item = kPairs pairs of columns of every row: a 16-byte vector for fp32 storage (4 columns), HALF a vector for
+// bf16 storage (8 bytes, 4 columns).  With whole bf16 vectors the per-thread state (five packed quantities per pair and
+// the loads in flight) takes 108 registers, two CTAs fit an SM and the pass is latency-bound at 5.8 TB/s; with half
+// vectors and eight Workers in flight it takes about 60 and four CTAs fit.
 template <typename T>
-__device__ __forceinline__ f32x2 pair_of(const uint4& v, int p);
+struct CombineItem {
+    static constexpr int kPairs = 2;
+    static constexpr int kCols = 4;
+    static constexpr int kUnroll = sizeof(T) == 2 ? 8 : 4;  // Workers whose loads are in flight together
+    // pair p (0 or 1) of the item as two floats
+    static __device__ __forceinline__ f32x2 pair(const uint2& lo, const uint2& hi, int p);
+};
 template <>
-__device__ __forceinline__ f32x2 pair_of<float>(const uint4& v, int p) {
-    return p == 0 ? pk(__uint_as_float(v.x), __uint_as_float(v.y)) : pk(__uint_as_float(v.z), __uint_as_float(v.w));
+__device__ __forceinline__ f32x2 CombineItem<float>::pair(const uint2& lo, const uint2& hi, int p) {
+    return p == 0 ? pk(__uint_as_float(lo.x), __uint_as_float(lo.y)) : pk(__uint_as_float(hi.x), __uint_as_float(hi.y));
 }
 template <>
-__device__ __forceinline__ f32x2 pair_of<__nv_bfloat16>(const uint4& v, int p) {
-    const uint32_t w = p == 0 ? v.x : p == 1 ? v.y : p == 2 ? v.z : v.w;
+__device__ __forceinline__ f32x2 CombineItem<__nv_bfloat16>::pair(const uint2& lo, const uint2&, int p) {
+    const uint32_t w = p == 0 ? lo.x : lo.y;
     return pk(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+// the item's bytes: 16 (fp32: lo and hi) or 8 (bf16: lo only)
+template <typename T>
+__device__ __forceinline__ void load_item(const T* p, uint2& lo, uint2& hi) {
+    if (sizeof(T) == 4) {
+        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(lo.x), "=r"(lo.y), "=r"(hi.x), "=r"(hi.y) : "l"(p));
+    } else {
+        asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(lo.x), "=r"(lo.y) : "l"(p));
+        hi = make_uint2(0, 0);
+    }
 }
 
 template <typename T>
 __global__ void __launch_bounds__(kCombineThreads)
 combine_vec_kernel(const T* __restrict__ theta, const T* __restrict__ g, int64_t n, int m,
                    const qn_coef_block* __restrict__ coef, T* __restrict__ out, const T* __restrict__ base) {
-    constexpr int kCols = Storage<T>::kVec;
-    constexpr int kPairs = kCols / 2;
+    using Item = CombineItem<T>;
+    constexpr int kCols = Item::kCols, kPairs = Item::kPairs, kUnroll = Item::kUnroll;
     __shared__ float c_sh[QN_MAX_M];
     if (threadIdx.x < QN_MAX_M) c_sh[threadIdx.x] = coef->c[threadIdx.x];
     const float tau = coef->tau, inv_m = coef->inv_m;
@@ -171,31 +190,33 @@ combine_vec_kernel(const T* __restrict__ theta, const T* __restrict__ g, int64_t
         const int64_t i0 = item * kCols;
         f32x2 th0[kPairs], g0[kPairs], sth[kPairs], sg[kPairs], acc[kPairs];
         {
-            const uint4 a = ldg_stream16(theta + i0), b = ldg_stream16(g + i0);
+            uint2 al, ah, bl, bh;
+            load_item(theta + i0, al, ah);
+            load_item(g + i0, bl, bh);
 #pragma unroll
             for (int p = 0; p < kPairs; ++p) {
-                th0[p] = sth[p] = pair_of<T>(a, p);
-                g0[p] = sg[p] = pair_of<T>(b, p);
+                th0[p] = sth[p] = Item::pair(al, ah, p);
+                g0[p] = sg[p] = Item::pair(bl, bh, p);
                 acc[p] = pk(0.f, 0.f);
             }
         }
-        for (int k = 1; k < m; k += kCombineUnroll) {
-            uint4 a[kCombineUnroll], b[kCombineUnroll];
+        for (int k = 1; k < m; k += kUnroll) {
+            uint2 al[kUnroll], ah[kUnroll], bl[kUnroll], bh[kUnroll];
 #pragma unroll
-            for (int u = 0; u < kCombineUnroll; ++u) {
+            for (int u = 0; u < kUnroll; ++u) {
                 if (k + u < m) {
-                    a[u] = ldg_stream16(theta + (int64_t)(k + u) * n + i0);
-                    b[u] = ldg_stream16(g + (int64_t)(k + u) * n + i0);
+                    load_item(theta + (int64_t)(k + u) * n + i0, al[u], ah[u]);
+                    load_item(g + (int64_t)(k + u) * n + i0, bl[u], bh[u]);
                 }
             }
 #pragma unroll
-            for (int u = 0; u < kCombineUnroll; ++u) {
+            for (int u = 0; u < kUnroll; ++u) {
                 if (k + u < m) {
                     const float ck = c_sh[k + u];
                     const f32x2 ck2 = pk(ck, ck);
 #pragma unroll
                     for (int p = 0; p < kPairs; ++p) {
-                        const f32x2 t = pair_of<T>(a[u], p), gg = pair_of<T>(b[u], p);
+                        const f32x2 t = Item::pair(al[u], ah[u], p), gg = Item::pair(bl[u], bh[u], p);
                         sth[p] = add2(sth[p], t);
                         sg[p] = add2(sg[p], gg);
                         acc[p] = fma2(ck2, sub2(sub2(gg, g0[p]), sub2(t, th0[p])), acc[p]);
@@ -208,11 +229,20 @@ combine_vec_kernel(const T* __restrict__ theta, const T* __restrict__ g, int64_t
 #pragma unroll
         for (int p = 0; p < kPairs; ++p) unpk(fma2(tm2, sg[p], fma2(sth[p], im2, acc[p])), res[2 * p], res[2 * p + 1]);
         if (base) {  // Eq. (4) applied to z: the correction is added to z instead of to the means
-            const uint4 zv = ldg_stream16(base + i0);
+            uint2 zl, zh;
+            load_item(base + i0, zl, zh);
 #pragma unroll
-            for (int p = 0; p < kPairs; ++p) unpk(add2(pair_of<T>(zv, p), acc[p]), res[2 * p], res[2 * p + 1]);
+            for (int p = 0; p < kPairs; ++p) unpk(add2(Item::pair(zl, zh, p), acc[p]), res[2 * p], res[2 * p + 1]);
         }
-        stg_stream16(out + i0, Storage<T>::pack(res));
+        if (sizeof(T) == 4) {
+            stg_stream16(out + i0, make_uint4(__float_as_uint(res[0]), __float_as_uint(res[1]), __float_as_uint(res[2]),
+                                              __float_as_uint(res[3])));
+        } else {
+            uint32_t w0, w1;  // cvt.rn.bf16x2.f32 d, a, b: a -> upper half, b -> lower half
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w0) : "f"(res[1]), "f"(res[0]));
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w1) : "f"(res[3]), "f"(res[2]));
+            asm volatile("st.global.cs.v2.u32 [%0], {%1,%2};" ::"l"(out + i0), "r"(w0), "r"(w1) : "memory");
+        }
     }
 }
 
@@ -222,7 +252,7 @@ static cudaError_t launch_combine_t(const T* theta, const T* g, int64_t n, int m
     const bool aligned = (reinterpret_cast<uintptr_t>(theta) % 16 == 0) && (reinterpret_cast<uintptr_t>(g) % 16 == 0) &&
                          (reinterpret_cast<uintptr_t>(out) % 16 == 0) && (reinterpret_cast<uintptr_t>(base) % 16 == 0) &&
                          ((n * (int64_t)sizeof(T)) % 16 == 0);
-    const int64_t nitems = aligned ? n / Storage<T>::kVec : n;
+    const int64_t nitems = aligned ? n / CombineItem<T>::kCols : n;
     const int64_t want = (nitems + kCombineThreads - 1) / kCombineThreads;
     int per_sm = 1;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, combine_vec_kernel<T>, kCombineThreads, 0) != cudaSuccess ||
