@@ -179,11 +179,12 @@ gram_direct_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict
 
 // ------------------------------------------------------------------------------------------------
 // Direct kernel fed by bulk copies, m <= 8, fast arithmetic mode, rows on 16-byte boundaries.  One thread
-// issues untiled TMA loads of 3.5 KB row segments into a ring of shared-memory stages (all m rows of
-// 1792 bf16 / 896 fp32 columns per stage, 196 KB in flight per SM), so the seven warps that do the
-// arithmetic never wait on HBM latency themselves; the register-fed kernel above reaches 5.3 TB/s with fp32
-// storage, this one 6.0.  Used for fp32 storage (see qn_launch_gram).  The arithmetic is kFast's, on packed pairs
-// of columns.
+// issues untiled TMA loads of 3.5 KB row segments into a ring of shared-memory stages (eight segments per
+// stage: 8 / MR column blocks of MR rows, 196 KB in flight per SM whatever m), so the seven warps that do the
+// arithmetic never wait on HBM latency themselves.  The arithmetic is kFast's on packed pairs of columns, for
+// MR = 2, 4 or 8 >= m rows.  Measured against the register-fed kernel above (TB/s): fp32 storage m = 8: 6.4 vs 5.3,
+// m = 4: 5.9 vs 3.2; bf16 storage m = 8: 4.5 vs 4.3, m = 4: 4.9 vs 2.4, m = 2: 4.5 vs 1.2 (with bf16 storage and
+// eight rows the pass is bound by the instructions per element).
 // Every wait is bounded; on a time-out the partial is poisoned and the error word set.
 // ------------------------------------------------------------------------------------------------
 // packed pairs of fp32 (one 64-bit register, two lanes of the fp32 pipe per instruction)
@@ -225,6 +226,32 @@ __device__ __forceinline__ uint64_t gs_pair<__nv_bfloat16>(const uint4& v, int q
     return gs_pk2(w << 16, w & 0xffff0000u);
 }
 
+// whether entry e of the 8-row packed layout (36 Gram entries by rows, then 8 products with the reference) involves
+// only rows < mr
+__host__ __device__ constexpr bool gs_used(int e, int mr) {
+    if (e >= kDirectTri) return e - kDirectTri < mr;
+    int k = 0, rem = e;
+    while (rem >= kDirectM - k) {
+        rem -= kDirectM - k;
+        ++k;
+    }
+    return k + rem < mr;
+}
+
+// the same for all 44 entries as a bit mask (a compile-time constant per mr)
+__host__ __device__ constexpr uint64_t gs_used_mask(int mr) {
+    uint64_t mask = 0;
+    for (int e = 0; e < kDirectAcc; ++e) mask |= (uint64_t)(gs_used(e, mr) ? 1 : 0) << e;
+    return mask;
+}
+
+// bytes of a row segment that starts at column c and has at most seg_cols columns (0 past the end of the row)
+template <typename T>
+__host__ __device__ inline uint32_t gs_block_bytes(int64_t n, int64_t c, int seg_cols) {
+    const int64_t left = n - c;
+    return left <= 0 ? 0u : (uint32_t)((left < seg_cols ? left : seg_cols) * (int64_t)sizeof(T));
+}
+
 constexpr int kGsWarps = 7;                   // warps that do the arithmetic; one more issues the loads: 256 threads,
 constexpr int kGsThreads = (kGsWarps + 1) * 32;  // so that every thread can have the registers its 132 sums need
 constexpr int kGsSeg = kGsWarps * 32 * 16;    // bytes of one row in a stage: one 16-byte vector per arithmetic thread
@@ -238,13 +265,19 @@ struct GsSmem {
     int abort;
 };
 
-template <typename T>
+// MR = 2, 4 or 8 >= m: the rows that are computed (the sums of rows >= MR stay zero and cost nothing; with MR = 8 for
+// every m the pass would be bound by the same instruction count whatever m, e.g. 2.3 TB/s at m = 4 with bf16 storage).
+// The sums keep their place in the 8-row packed layout, so the reduction is shared with the register-fed kernel.
+template <typename T, int MR>
 __global__ void __launch_bounds__(kGsThreads, 1)
 gram_stream_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ partials, int* __restrict__ error_word) {
     constexpr int kCols = Storage<T>::kVec;
-    constexpr int kTileCols = kGsSeg / (int)sizeof(T);
+    constexpr int kSegCols = kGsSeg / (int)sizeof(T);   // columns of one row segment
+    constexpr int NB = kDirectM / MR;                    // a stage's 8 segments hold NB column blocks of MR rows, so that
+    constexpr int kTileCols = NB * kSegCols;             // every m keeps the same number of bytes in flight
     // each half of a packed accumulator sums every other column: kFlushCols columns per half between flushes
     constexpr int kFlushIters = 2 * kFlushCols / kCols;
+    constexpr uint64_t kUsed = gs_used_mask(MR);  // the sums this instance forms
     extern __shared__ unsigned char smem_raw[];
     GsSmem& sm = *reinterpret_cast<GsSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -273,10 +306,18 @@ gram_stream_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict
                 const int s = it % kGsStages, use = it / kGsStages;
                 if (use > 0) mbar_wait(&sm.empty[s], (uint32_t)((use - 1) & 1), abort);
                 const int64_t col0 = (blockIdx.x + (int64_t)it * gridDim.x) * kTileCols;
-                const int64_t left = n - col0;
-                const uint32_t bytes = (uint32_t)((left < kTileCols ? left : kTileCols) * (int64_t)sizeof(T));
-                mbar_arrive_expect_tx(&sm.full[s], (uint32_t)m * bytes);
-                for (int k = 0; k < m; ++k) bulk_load(sm.seg[s][k], g + (int64_t)k * n + col0, bytes, &sm.full[s]);
+                uint32_t total = 0;
+#pragma unroll
+                for (int b = 0; b < NB; ++b) total += gs_block_bytes<T>(n, col0 + (int64_t)b * kSegCols, kSegCols);
+                mbar_arrive_expect_tx(&sm.full[s], (uint32_t)m * total);
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    const int64_t c = col0 + (int64_t)b * kSegCols;
+                    const uint32_t bytes = gs_block_bytes<T>(n, c, kSegCols);
+                    if (bytes)
+                        for (int k = 0; k < m; ++k)
+                            bulk_load(sm.seg[s][b * MR + k], g + (int64_t)k * n + c, bytes, &sm.full[s]);
+                }
             }
         }
     } else {
@@ -292,51 +333,64 @@ gram_stream_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict
         int iters = 0;
         for (int it = 0; it < my_tiles; ++it) {
             const int s = it % kGsStages, use = it / kGsStages;
-            const int64_t left = n - (blockIdx.x + (int64_t)it * gridDim.x) * kTileCols;
-            const uint32_t bytes = (uint32_t)((left < kTileCols ? left : kTileCols) * (int64_t)sizeof(T));
+            const int64_t col0 = (blockIdx.x + (int64_t)it * gridDim.x) * kTileCols;
             const bool ok = mbar_wait(&sm.full[s], (uint32_t)(use & 1), abort);
-            const bool live = ok && (uint32_t)(tid * 16) < bytes;  // the last tile may be short
-            uint4 v[kDirectM];
+            uint4 vall[kDirectM];  // segment b * MR + k: row k of column block b
 #pragma unroll
-            for (int k = 0; k < kDirectM; ++k) {
-                v[k] = make_uint4(0, 0, 0, 0);
-                if (live && k < m) v[k] = *reinterpret_cast<const uint4*>(sm.seg[s][k] + tid * 16);
+            for (int b = 0; b < NB; ++b) {
+                // the last tile may be short or end before this block
+                const bool live = ok && (uint32_t)(tid * 16) < gs_block_bytes<T>(n, col0 + (int64_t)b * kSegCols, kSegCols);
+#pragma unroll
+                for (int k = 0; k < MR; ++k) {
+                    vall[b * MR + k] = make_uint4(0, 0, 0, 0);
+                    if (live && k < m) vall[b * MR + k] = *reinterpret_cast<const uint4*>(sm.seg[s][b * MR + k] + tid * 16);
+                }
             }
             // the values are in registers: the stage can be refilled
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.empty[s]);
 #pragma unroll
-            for (int q = 0; q < kCols / 2; ++q) {
-                uint64_t x[kDirectM];
+            for (int b = 0; b < NB; ++b) {
+            const uint4* v = vall + b * MR;
 #pragma unroll
-                for (int k = 0; k < kDirectM; ++k) x[k] = gs_pair<T>(v[k], q);
+            for (int q = 0; q < kCols / 2; ++q) {
+                uint64_t x[MR];
+#pragma unroll
+                for (int k = 0; k < MR; ++k) x[k] = gs_pair<T>(v[k], q);
                 uint64_t sum = x[0];
 #pragma unroll
-                for (int k = 1; k < kDirectM; ++k) sum = gs_add2(sum, x[k]);
+                for (int k = 1; k < MR; ++k) sum = gs_add2(sum, x[k]);
                 const uint64_t r = gs_mul2(sum, inv_m2);
+                // padding rows (m <= k < MR) read as zero and become -r here: they only reach sums that are never output
 #pragma unroll
-                // padding rows (k >= m) read as zero and become -r here: they only reach sums that are never output
-                for (int k = 0; k < kDirectM; ++k) x[k] = gs_sub2(x[k], r);
+                for (int k = 0; k < MR; ++k) x[k] = gs_sub2(x[k], r);
 #pragma unroll
-                for (int k = 0, idx = 0; k < kDirectM; ++k) {
+                for (int k = 0; k < MR; ++k) {
 #pragma unroll
-                    for (int l = k; l < kDirectM; ++l, ++idx) acc[idx] = gs_fma2(x[k], x[l], acc[idx]);
+                    for (int l = k; l < MR; ++l) {
+                        const int idx = k * kDirectM - (k * (k - 1)) / 2 + (l - k);  // place in the 8-row packed layout
+                        acc[idx] = gs_fma2(x[k], x[l], acc[idx]);
+                    }
                 }
 #pragma unroll
-                for (int k = 0; k < kDirectM; ++k) acc[kDirectTri + k] = gs_fma2(x[k], r, acc[kDirectTri + k]);
+                for (int k = 0; k < MR; ++k) acc[kDirectTri + k] = gs_fma2(x[k], r, acc[kDirectTri + k]);
             }
             if (++iters == kFlushIters) {
                 iters = 0;
 #pragma unroll
                 for (int e = 0; e < kDirectAcc; ++e) {
-                    acc64[e] += (double)__uint_as_float((uint32_t)acc[e]) + (double)__uint_as_float((uint32_t)(acc[e] >> 32));
-                    acc[e] = 0ull;
+                    if ((kUsed >> e) & 1ull) {
+                        acc64[e] += (double)__uint_as_float((uint32_t)acc[e]) + (double)__uint_as_float((uint32_t)(acc[e] >> 32));
+                        acc[e] = 0ull;
+                    }
                 }
             }
+            }  // column blocks of the stage
         }
 #pragma unroll
         for (int e = 0; e < kDirectAcc; ++e)
-            acc64[e] += (double)__uint_as_float((uint32_t)acc[e]) + (double)__uint_as_float((uint32_t)(acc[e] >> 32));
+            if ((kUsed >> e) & 1ull)
+                acc64[e] += (double)__uint_as_float((uint32_t)acc[e]) + (double)__uint_as_float((uint32_t)(acc[e] >> 32));
     }
     __syncthreads();
     if (*abort) {
@@ -353,13 +407,14 @@ gram_stream_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict
 template <typename T>
 static cudaError_t launch_gram_stream(const T* g, int64_t n, int m, double* partials, int* num_partials,
                                       int max_partials, int* error_word, cudaStream_t st) {
-    const int64_t tile_cols = kGsSeg / (int64_t)sizeof(T);
+    const int mr = m <= 2 ? 2 : m <= 4 ? 4 : 8;
+    const int64_t tile_cols = (kDirectM / mr) * (kGsSeg / (int64_t)sizeof(T));
     const int64_t ntiles = (n + tile_cols - 1) / tile_cols;
     const int sms = qn_sm_count();
     int grid = (int)(ntiles < sms ? ntiles : sms);
     if (grid > max_partials) grid = max_partials;
     *num_partials = grid;
-    auto kern = gram_stream_kernel<T>;
+    auto kern = m <= 2 ? gram_stream_kernel<T, 2> : m <= 4 ? gram_stream_kernel<T, 4> : gram_stream_kernel<T, 8>;
     const size_t smem = sizeof(GsSmem) + 128;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -598,25 +653,15 @@ static bool tc_allowed() {
     const char* v = getenv("QN_GRAM_PATH");
     return !(v && v[0] == 'a');
 }
-// QN_GRAM_PATH=stream sends bf16 storage to the bulk-copy direct kernel as well (A/B measurements)
-static bool stream_forced() {
-    const char* v = getenv("QN_GRAM_PATH");
-    return v && v[0] == 's';
-}
-
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
                            int* num_partials, int max_partials, cudaStream_t st, int* launches, int* error_word) {
     cudaError_t e;
     const int64_t elem = dtype == QN_F32 ? 4 : 2;
     if (!raw && tc_allowed() && qn_gram_tc_applicable(dtype, g, n, m)) {
         e = qn_launch_gram_tc(dtype, g, n, m, partials, num_partials, max_partials, error_word, st);
-    } else if (!raw && tc_allowed() && (dtype == QN_F32 || m == qn::kDirectM || stream_forced()) && m <= qn::kDirectM &&
-               n >= QN_PRECISE_BELOW && reinterpret_cast<uintptr_t>(g) % 16 == 0 && (n * elem) % 16 == 0) {
-        // Bulk-copy variant of the direct kernel (QN_GRAM_PATH=alu keeps the register-fed one, QN_GRAM_PATH=stream
-        // forces this one, for A/B runs).  Measured: fp32 storage 6.4 TB/s at m = 8 and 4.9 at m = 5 against 5.3 and
-        // 3.8 register-fed; bf16 storage 4.5 against 4.3 at m = 8 but 2.3 against 2.4 at m = 4 (with bf16 both are
-        // bound by the instructions per element, which do not shrink with m because all eight rows are always
-        // computed), so bf16 storage comes here only with eight Workers.
+    } else if (!raw && tc_allowed() && m <= qn::kDirectM && n >= QN_PRECISE_BELOW &&
+               reinterpret_cast<uintptr_t>(g) % 16 == 0 && (n * elem) % 16 == 0) {
+        // bulk-copy variant of the direct kernel (QN_GRAM_PATH=alu keeps the register-fed one, for A/B runs)
         e = dtype == QN_F32 ? qn::launch_gram_stream(static_cast<const float*>(g), n, m, partials, num_partials,
                                                      max_partials, error_word, st)
                             : qn::launch_gram_stream(static_cast<const __nv_bfloat16*>(g), n, m, partials,

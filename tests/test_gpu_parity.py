@@ -352,6 +352,20 @@ def test_argument_validation(qn):
     assert L.qn_push(hd.ptr, -2, o.data_ptr(), o.data_ptr(), st) == qn.QN_ERR_INVALID
     assert L.qn_rebuild(hd.ptr, st) == qn.QN_ERR_STATE
     assert L.qn_update_window(hd.ptr, 1.0, 0.1, o.data_ptr(), None, None, st) == qn.QN_ERR_STATE
+    # the entry points added around the step: same checks
+    gram = torch.zeros(4 * 4 + 4, dtype=torch.float64, device="cuda")
+    z = torch.zeros(1000, device="cuda")
+    tp, op, zp, gp = t.data_ptr(), o.data_ptr(), z.data_ptr(), gram.data_ptr()
+    assert L.qn_update_from_gram(hd.ptr, tp, tp, None, 1.0, 0.1, op, None, None, st) == qn.QN_ERR_INVALID
+    assert L.qn_update_from_gram(hd.ptr, tp, tp, gp, 1.0, 0.0, op, None, None, st) == qn.QN_ERR_INVALID
+    assert L.qn_update_from_gram(hd.ptr, tp, tp, gp, 1.0, 0.1, tp + 64, None, None, st) == qn.QN_ERR_INVALID
+    assert L.qn_apply_hinv(hd.ptr, tp, tp, 0.1, None, op, None, None, st) == qn.QN_ERR_INVALID
+    assert L.qn_apply_hinv(hd.ptr, tp, tp, -0.1, zp, op, None, None, st) == qn.QN_ERR_INVALID
+    assert L.qn_apply_hinv(hd.ptr, tp, tp, 0.1, zp, zp, None, None, st) == qn.QN_ERR_INVALID  # out overlaps z
+    assert L.qn_apply_hinv(hd.ptr, tp, tp, 0.1, zp, tp, None, None, st) == qn.QN_ERR_INVALID  # out overlaps theta
+    assert L.qn_set_rank_cap(None, 1) == qn.QN_ERR_INVALID
+    assert L.qn_set_tau_cap(None, 1) == qn.QN_ERR_INVALID
+    assert L.qn_set_rank_cap(hd.ptr, 2) == qn.QN_OK and L.qn_set_rank_cap(hd.ptr, -5) == qn.QN_OK
     assert L.qn_status_sync(hd.ptr) == qn.QN_OK
     hd.close()
 
@@ -479,15 +493,19 @@ def test_sharded_step_matches_the_whole_problem(qn, dtype, m, n, shards):
 
 # --------------------------------------------------------------------------- bulk-copy Gram path (n >= 2^22, m <= 8)
 @pytest.mark.parametrize("dtype,m,n,gap", [
-    ("bf16", 8, (1 << 22) + 8 * 3, True),    # config 4's first sweep point (register-fed kernel, fast mode)
+    ("bf16", 8, (1 << 22) + 8 * 3, True),    # config 4's first sweep point: short last tile
     ("bf16", 8, 1 << 22, False),
-    ("f32", 5, (1 << 22) + 4, True),         # bulk-copy kernel: three padding rows, short last tile
+    ("f32", 5, (1 << 22) + 4, True),         # three padding rows, short last tile
     ("f32", 8, 1 << 22, True),
     ("f32", 8, 1 << 22, False),
+    ("bf16", 4, 1 << 22, False),             # four rows computed
+    ("f32", 3, (1 << 22) + 8, False),
+    ("bf16", 2, 1 << 22, False),             # two rows computed
+    ("f32", 1, 1 << 22, False),              # one Worker: sigma = 0, the plain step
 ])
 def test_direct_gram_paths_at_large_n(qn, dtype, m, n, gap):
-    """Above 2^22 columns and with at most 8 Workers: fp32 storage on aligned rows is fed by bulk copies into
-    shared-memory stages, bf16 storage by register prefetch.  Same bar as everywhere."""
+    """Above 2^22 columns and with at most 8 Workers on aligned rows the Gram pass is fed by bulk copies into
+    shared-memory stages and computes 2, 4 or 8 rows.  Same bar as everywhere."""
     cfg = W.Config(41, n, m, dtype, -2, 2, 0, 0.01, 1e-4, 1.0, 0.01)
     lam = 0.05 if (gap and dtype == "bf16") else 0.01
     theta, g = W.generate(cfg, "cuda", gap_lam=lam if gap else None, gap_scale=1.0 if (gap and dtype == "bf16") else None)
