@@ -396,6 +396,7 @@ gram_stream_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict
     if (*abort) {
         // a wait ran out: give bulk copies that may still be in flight into this CTA's shared memory time to land
         // (bounded: about a millisecond), report, and poison the partial so that the solve sees the failure
+#pragma unroll 1
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
         if (tid == 0 && error_word) atomicExch(error_word, 1);
 #pragma unroll
@@ -424,14 +425,14 @@ static cudaError_t launch_gram_stream(const T* g, int64_t n, int m, double* part
 
 // ------------------------------------------------------------------------------------------------
 // Tiled kernel, 9 <= m <= 64, plain fp32 ALUs.  A tile of kTileCols columns is staged in shared
-// memory as shifted fp32 values, one record of RBP floats per column: rows 0..m-1 = x_k, row m =
-// the reference r (so that entry (k, m) of the extended Gram is t_k), zero padding up to a
-// multiple of 8.  The extended Gram is cut into 8x8 blocks; a thread owns one upper-triangle block
-// and a fixed residue class of the tile's columns, with the 64 accumulators in registers.
+// memory as shifted fp32 values, one record of RBP floats per column: rows 0..m-1 = x_k, zero padding up
+// to a multiple of 8 (RB rows), then the reference r of the column.  The Gram is cut into 8x8 blocks; a
+// thread owns one upper-triangle block and a fixed residue class of the tile's columns, with the 64
+// accumulators in registers, plus eight for t_k = sum_i x_k r, which the diagonal blocks deliver.
 // ------------------------------------------------------------------------------------------------
 constexpr int kTileCols = 128;
-constexpr int kMaxBlocks = (QN_MAX_M + 1 + 7) / 8;                 // 9
-constexpr int kMaxRBP = 8 * kMaxBlocks + 4;                        // 76 floats per column record
+constexpr int kMaxBlocks = (QN_MAX_M + 7) / 8;                     // 8
+constexpr int kMaxRBP = 8 * kMaxBlocks + 4;                        // 68 floats per column record
 
 struct TiledSmem {
     float xs[kTileCols * kMaxRBP];
@@ -448,12 +449,12 @@ gram_tiled_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict_
     constexpr int kColGroups = kTileCols / kCols;           // load items per row per tile
     constexpr int kRowGroups = kThreads / kColGroups;       // 8 (fp32 x4), 16 (bf16 x8), 2 (scalar)
 
-    const int nb = (m + 1 + 7) / 8;
+    const int nb = (m + 7) / 8;
     const int RB = 8 * nb;
-    const int RBP = RB + 4;
+    const int RBP = RB + 4;  // the record's entry RB holds the reference r of the column
     const int ntile = nb * (nb + 1) / 2;
-    int S = 8;
-    while (S < ntile) S <<= 1;  // slots per column step: 8, 16, 32 or 64
+    int S = 4;
+    while (S < ntile) S <<= 1;  // slots per column step: 4, 8, 16, 32 or 64
     const int slot = threadIdx.x % S;
     const int col0 = threadIdx.x / S;
     const int colstep = kThreads / S;
@@ -479,33 +480,70 @@ gram_tiled_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict_
         acc[e] = 0.f;
         acc64[e] = 0.0;
     }
+    // t_k = sum_i x_k r: eight more sums, meaningful in the threads of the diagonal blocks (ta == tb)
+    float tacc[8];
+    double tacc64[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        tacc[e] = 0.f;
+        tacc64[e] = 0.0;
+    }
     const float inv_m = 1.0f / (float)m;
     const int rg = threadIdx.x % kRowGroups, cg = threadIdx.x / kRowGroups;
     const int64_t ntiles = (n + kTileCols - 1) / kTileCols;
     int cols_since_flush = 0;
 
-    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    // This thread's part of a tile (rows rg, rg + kRowGroups, ... of its column group) is fetched one tile ahead
+    // into registers, so that the latency of the loads is hidden behind the previous tile's arithmetic (the fp64
+    // modes, which run at small n where little else hides it; the fast mode has no registers to spare for it).
+    constexpr bool kAhead = kMode != kFast;
+    constexpr int kPre = QN_MAX_M / kRowGroups;
+    constexpr int kPreWords = kAligned ? 4 : 1;  // a 16-byte vector, or one element as fp32
+    uint32_t pre[kPre][kPreWords];
+    auto fetch = [&](int64_t tile) {
         const int64_t i0 = tile * kTileCols + (int64_t)cg * kCols;
+#pragma unroll
+        for (int j = 0; j < kPre; ++j) {
+            const int k = rg + j * kRowGroups;
+#pragma unroll
+            for (int w = 0; w < kPreWords; ++w) pre[j][w] = 0u;
+            if (k < m && tile < ntiles && i0 < n) {
+                if (kAligned) {
+                    const uint4 v = ldg_stream16(g + (int64_t)k * n + i0);
+                    pre[j][0] = v.x;
+                    pre[j][kPreWords > 1 ? 1 : 0] = v.y;
+                    pre[j][kPreWords > 2 ? 2 : 0] = v.z;
+                    pre[j][kPreWords > 3 ? 3 : 0] = v.w;
+                } else {
+                    pre[j][0] = __float_as_uint(Storage<T>::load1(g + (int64_t)k * n + i0));
+                }
+            }
+        }
+    };
+    if (kAhead) fetch(blockIdx.x);
+
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        if (!kAhead) fetch(tile);
         // pass A: raw values into the column records, partial sums over this thread's rows
         float ps[kCols];
 #pragma unroll
         for (int e = 0; e < kCols; ++e) ps[e] = 0.f;
-        for (int k = rg; k < m; k += kRowGroups) {
-            float val[kCols];
-            if (kAligned) {
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (i0 < n) v = ldg_stream16(g + (int64_t)k * n + i0);
 #pragma unroll
-                for (int e = 0; e < kCols; ++e) val[e] = Storage<T>::get(v, e);
-            } else {
-                val[0] = i0 < n ? Storage<T>::load1(g + (int64_t)k * n + i0) : 0.f;
-            }
+        for (int j = 0; j < kPre; ++j) {
+            const int k = rg + j * kRowGroups;
+            if (k < m) {
 #pragma unroll
-            for (int e = 0; e < kCols; ++e) {
-                sm.xs[(cg * kCols + e) * RBP + k] = val[e];
-                ps[e] += val[e];
+                for (int e = 0; e < kCols; ++e) {
+                    const float val = kAligned ? Storage<T>::get(make_uint4(pre[j][0], pre[j][kPreWords > 1 ? 1 : 0],
+                                                                            pre[j][kPreWords > 2 ? 2 : 0],
+                                                                            pre[j][kPreWords > 3 ? 3 : 0]), e)
+                                               : __uint_as_float(pre[j][0]);
+                    sm.xs[(cg * kCols + e) * RBP + k] = val;
+                    ps[e] += val;
+                }
             }
         }
+        if (kAhead) fetch(tile + gridDim.x);
 #pragma unroll
         for (int e = 0; e < kCols; ++e) sm.psum[(cg * kCols + e) * (kRowGroups + 1) + rg] = ps[e];
         __syncthreads();
@@ -526,8 +564,8 @@ gram_tiled_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict_
         if (rg == 0) {
 #pragma unroll
             for (int e = 0; e < kCols; ++e) {
-                sm.xs[(cg * kCols + e) * RBP + m] = r[e];
-                for (int k = m + 1; k < RB; ++k) sm.xs[(cg * kCols + e) * RBP + k] = 0.f;
+                sm.xs[(cg * kCols + e) * RBP + RB] = r[e];
+                for (int k = m; k < RB; ++k) sm.xs[(cg * kCols + e) * RBP + k] = 0.f;
             }
         }
         __syncthreads();
@@ -539,11 +577,14 @@ gram_tiled_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict_
                 const float4 b0 = rec[2 * tb], b1 = rec[2 * tb + 1];
                 const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
                 const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                const float rc = sm.xs[c * RBP + RB];
                 if (kMode == kFast) {
 #pragma unroll
                     for (int p = 0; p < 8; ++p)
 #pragma unroll
                         for (int q = 0; q < 8; ++q) acc[p * 8 + q] = fmaf(a[p], b[q], acc[p * 8 + q]);
+#pragma unroll
+                    for (int p = 0; p < 8; ++p) tacc[p] = fmaf(a[p], rc, tacc[p]);
                 } else {
                     double ad[8], bd[8];
 #pragma unroll
@@ -555,6 +596,9 @@ gram_tiled_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict_
                     for (int p = 0; p < 8; ++p)
 #pragma unroll
                         for (int q = 0; q < 8; ++q) acc64[p * 8 + q] = fma(ad[p], bd[q], acc64[p * 8 + q]);
+                    const double rd = (double)rc;
+#pragma unroll
+                    for (int p = 0; p < 8; ++p) tacc64[p] = fma(ad[p], rd, tacc64[p]);
                 }
             }
         }
@@ -567,6 +611,11 @@ gram_tiled_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict_
                     acc64[e] += (double)acc[e];
                     acc[e] = 0.f;
                 }
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    tacc64[e] += (double)tacc[e];
+                    tacc[e] = 0.f;
+                }
             }
         }
         __syncthreads();
@@ -574,6 +623,8 @@ gram_tiled_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict_
     if (kMode == kFast) {
 #pragma unroll
         for (int e = 0; e < 64; ++e) acc64[e] += (double)acc[e];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) tacc64[e] += (double)tacc[e];
     }
 
     // CTA reduction: for each block, sum the kThreads/S column classes in the order 0,1,2,...
@@ -592,13 +643,21 @@ gram_tiled_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict_
             double s = 0.0;
             for (int q = 0; q < colstep; ++q) s += red[(q * S + sl) * 16 + (w % 16)];
             const int row = 8 * tile_a[sl] + e / 8, col = 8 * tile_b[sl] + e % 8;
-            if (row < m && row <= col) {
-                if (col < m)
-                    out[qn_tri_index(m, row, col)] = s;
-                else if (col == m)
-                    out[tri_len + row] = s;
-            }
+            if (row <= col && col < m) out[qn_tri_index(m, row, col)] = s;
         }
+    }
+    // t from the diagonal blocks, same fixed order
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < 8; ++e) red[threadIdx.x * 16 + e] = tacc64[e];
+    __syncthreads();
+    for (int w = threadIdx.x; w < S * 8; w += kThreads) {
+        const int sl = w / 8, e = w % 8;
+        if (sl >= ntile || tile_a[sl] != tile_b[sl]) continue;
+        double s = 0.0;
+        for (int q = 0; q < colstep; ++q) s += red[(q * S + sl) * 16 + e];
+        const int row = 8 * tile_a[sl] + e;
+        if (row < m) out[tri_len + row] = s;
     }
 }
 

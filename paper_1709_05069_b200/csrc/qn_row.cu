@@ -257,6 +257,7 @@ row_stream_kernel(const T* __restrict__ window_g, const T* __restrict__ g_col, T
     if (*abort) {
         // a wait ran out: give the bulk copies that may still be in flight into this CTA's shared memory time to
         // land (bounded: about a millisecond) before the CTA returns
+#pragma unroll 1
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
     }
     // CTA reduction in a fixed order, then last-CTA-done as in row_kernel
