@@ -16,18 +16,19 @@
 
 namespace qn {
 
-constexpr int kLd = QN_MAX_M + 1;  // leading dimension of the shared matrices (odd: no bank conflicts)
+constexpr int kLd = QN_MAX_M + 2;  // leading dimension of the shared matrices (even: 2x1 pairs of doubles are 16-byte aligned)
 constexpr int kMaxSweeps = 30;
 
 struct SolveSmem {
     double A[QN_MAX_M * kLd];
     double V[QN_MAX_M * kLd];  // also scratch for the partial sums before the Jacobi phase
+    double A2[QN_MAX_M * kLd], V2[QN_MAX_M * kLd];  // the Jacobi rounds read one copy and write the other
     double B[QN_MAX_M * kLd];  // reference-shifted Gram of theta (learning-rate cap only)
     double w[QN_MAX_M];
     double rowsum[QN_MAX_M];
     double mu[QN_MAX_M];
     double sigma[QN_MAX_M];
-    double rot_c[QN_MAX_M / 2], rot_s[QN_MAX_M / 2], rot_t[QN_MAX_M / 2];
+    double rot_c[QN_MAX_M / 2], rot_s[QN_MAX_M / 2];
     double modec[QN_MAX_M];
     double d[QN_MAX_M];
     double red[32];
@@ -50,21 +51,6 @@ __device__ __forceinline__ double block_sum(double x, double* red) {
     double s = 0.0;
     for (int i = 0; i < nw; ++i) s += red[i];
     return s;
-}
-
-// (p, q), p < q, of pair k in round r of the round-robin ordering over M2 (even) indices
-__device__ __forceinline__ void rr_pair(int M2, int r, int k, int& p, int& q) {
-    const int N = M2 - 1;
-    int a, b;
-    if (k == 0) {
-        a = N;
-        b = r;
-    } else {
-        a = (r + k) % N;
-        b = (r - k + N) % N;
-    }
-    p = a < b ? a : b;
-    q = a < b ? b : a;
 }
 
 __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
@@ -204,9 +190,16 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
     }
 
     // ---------------------------------------------------------------- phase 3: two-sided Jacobi
-    // Round-robin ordering: M2/2 disjoint pairs per round, M2-1 rounds per sweep.  Thread (a, b) owns
-    // the 2x2 block (rows of pair a) x (columns of pair b) for the round; the threads on the diagonal
-    // (a == b) first compute their pair's rotation and publish (c, s).  Two barriers per round.
+    // Round-robin ordering as a systolic array (Brent and Luk): the matrix is kept in the order of the tournament
+    // table, pair k = physical positions (2k, 2k+1), so thread (a, b) always owns the 2x2 block at rows 2a, 2a+1 and
+    // columns 2b, 2b+1, loads it with two 16-byte reads, and writes the rotated entries to where their rows and
+    // columns move for the next round (position 0 stays, the other top positions 2k move right, the bottom
+    // positions 2k+1 move left, the ends turn round).  M2-1 rounds per sweep bring every pair together once.  The
+    // rounds read one copy of A and V and write the other.  (With the blocks addressed through the changing index
+    // pairs instead, the scattered 8-byte accesses made the kernel shared-memory bound at about 1200 cycles per
+    // round.)  The threads on the diagonal (a == b) compute their pair's rotation and publish (c, s): two
+    // barriers per round.  The eigenvalues and the columns of V end up in tournament order, which phase 4 does
+    // not care about; a padding index (odd m) never rotates and keeps its zero eigenvalue.
     const int M2 = m + (m & 1);
     const int H = M2 / 2;
     const int N = M2 - 1;
@@ -230,9 +223,19 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
     const double inv_fro = fro > 0.0 ? 1.0 / fro : 0.0;  // brings entries into fp32 range whatever the data's scale
     const int pa_idx = tid / H, pb_idx = tid % H;
     const bool worker = tid < H * H;
-    // positions of this thread's two pairs in round 0; each round both members move one step round the circle
-    int a0 = pa_idx == 0 ? N : pa_idx % N, a1 = pa_idx == 0 ? 0 : (N - pa_idx) % N;
-    int b0 = pb_idx == 0 ? N : pb_idx % N, b1 = pb_idx == 0 ? 0 : (N - pb_idx) % N;
+    // where physical position i goes after a round
+    auto next_pos = [&](int i) -> int {
+        if (H == 1 || i == 0) return i;
+        if (i == 1) return 2;
+        if (i & 1) return i - 2;
+        return i == M2 - 2 ? M2 - 1 : i + 2;
+    };
+    const int ra = 2 * pa_idx, cb = 2 * pb_idx;  // this thread's block, every round
+    const int nr0 = next_pos(ra), nr1 = next_pos(ra + 1), nc0 = next_pos(cb), nc1 = next_pos(cb + 1);
+    double* Ar = sm.A;
+    double* Aw = sm.A2;
+    double* Vr = sm.V;
+    double* Vw = sm.V2;
     int sweeps = 0;
     bool converged = (fro == 0.0) || m < 2;
     // Rotation that zeroes a_pq.  The angle comes from fp32 arithmetic on values scaled into fp32 range
@@ -260,52 +263,57 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
     };
     while (!converged && sweeps < kMaxSweeps) {
         for (int r = 0; r < N; ++r) {
-            const int pa = a0 < a1 ? a0 : a1, qa = a0 < a1 ? a1 : a0;
-            const int pb = b0 < b1 ? b0 : b1, qb = b0 < b1 ? b1 : b0;
-            // the thread on the diagonal block of pair a computes that pair's rotation for everybody
-            if (worker && pa_idx == pb_idx) {
-                double c, s2;
-                rotation(sm.A[pa * kLd + pa], sm.A[qa * kLd + qa], sm.A[pa * kLd + qa], c, s2);
-                sm.rot_c[pa_idx] = c;
-                sm.rot_s[pa_idx] = s2;
+            double x00 = 0.0, x01 = 0.0, x10 = 0.0, x11 = 0.0;
+            if (worker) {
+                const double2 r0 = *reinterpret_cast<const double2*>(&Ar[ra * kLd + cb]);
+                const double2 r1 = *reinterpret_cast<const double2*>(&Ar[(ra + 1) * kLd + cb]);
+                x00 = r0.x;
+                x01 = r0.y;
+                x10 = r1.x;
+                x11 = r1.y;
+                if (pa_idx == pb_idx) {  // the diagonal block holds a_pp, a_pq, a_qq of pair a
+                    double c, s2;
+                    rotation(x00, x11, x01, c, s2);
+                    sm.rot_c[pa_idx] = c;
+                    sm.rot_s[pa_idx] = s2;
+                }
             }
             asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
             if (worker) {
                 const double ca = sm.rot_c[pa_idx], sa = sm.rot_s[pa_idx];
-                const double cb = sm.rot_c[pb_idx], sb = sm.rot_s[pb_idx];
-                const double x00 = sm.A[pa * kLd + pb], x01 = sm.A[pa * kLd + qb];
-                const double x10 = sm.A[qa * kLd + pb], x11 = sm.A[qa * kLd + qb];
-                const double v00 = sm.V[(2 * pa_idx) * kLd + pb], v01 = sm.V[(2 * pa_idx) * kLd + qb];
-                const double v10 = sm.V[(2 * pa_idx + 1) * kLd + pb], v11 = sm.V[(2 * pa_idx + 1) * kLd + qb];
-                // Y = J_a^T X J_b on this thread's 2x2 block (only this thread touches these four entries)
-                const double t00 = cb * x00 - sb * x01, t01 = sb * x00 + cb * x01;
-                const double t10 = cb * x10 - sb * x11, t11 = sb * x10 + cb * x11;
+                const double cbr = sm.rot_c[pb_idx], sbr = sm.rot_s[pb_idx];
+                const double2 v0 = *reinterpret_cast<const double2*>(&Vr[ra * kLd + cb]);
+                const double2 v1 = *reinterpret_cast<const double2*>(&Vr[(ra + 1) * kLd + cb]);
+                // Y = J_a^T X J_b on this thread's 2x2 block
+                const double t00 = cbr * x00 - sbr * x01, t01 = sbr * x00 + cbr * x01;
+                const double t10 = cbr * x10 - sbr * x11, t11 = sbr * x10 + cbr * x11;
                 double y00 = ca * t00 - sa * t10, y10 = sa * t00 + ca * t10;
                 double y01 = ca * t01 - sa * t11, y11 = sa * t01 + ca * t11;
                 if (pa_idx == pb_idx) y01 = y10 = 0.5 * (y01 + y10);  // keep the diagonal block symmetric
-                sm.A[pa * kLd + pb] = y00;
-                sm.A[pa * kLd + qb] = y01;
-                sm.A[qa * kLd + pb] = y10;
-                sm.A[qa * kLd + qb] = y11;
-                // V <- V J_b on rows 2*pa_idx, 2*pa_idx + 1
-                sm.V[(2 * pa_idx) * kLd + pb] = cb * v00 - sb * v01;
-                sm.V[(2 * pa_idx) * kLd + qb] = sb * v00 + cb * v01;
-                sm.V[(2 * pa_idx + 1) * kLd + pb] = cb * v10 - sb * v11;
-                sm.V[(2 * pa_idx + 1) * kLd + qb] = sb * v10 + cb * v11;
+                Aw[nr0 * kLd + nc0] = y00;
+                Aw[nr0 * kLd + nc1] = y01;
+                Aw[nr1 * kLd + nc0] = y10;
+                Aw[nr1 * kLd + nc1] = y11;
+                // V <- V J_b on rows 2a, 2a+1 (the rows of V are not reordered, its columns move with A's)
+                Vw[ra * kLd + nc0] = cbr * v0.x - sbr * v0.y;
+                Vw[ra * kLd + nc1] = sbr * v0.x + cbr * v0.y;
+                Vw[(ra + 1) * kLd + nc0] = cbr * v1.x - sbr * v1.y;
+                Vw[(ra + 1) * kLd + nc1] = sbr * v1.x + cbr * v1.y;
             }
             asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
-            // next round: every index except the fixed one (N) moves one step
-            if (a0 != N && ++a0 == N) a0 = 0;
-            if (++a1 == N) a1 = 0;
-            if (b0 != N && ++b0 == N) b0 = 0;
-            if (++b1 == N) b1 = 0;
+            double* t = Ar;
+            Ar = Aw;
+            Aw = t;
+            t = Vr;
+            Vr = Vw;
+            Vw = t;
         }
         ++sweeps;
         // converged when no off-diagonal element exceeds the threshold (one pass over the matrix)
         int big = 0;
         for (int e = tid; e < M2 * M2; e += jthreads) {
             const int k = e / M2, l = e % M2;
-            big |= (k != l) && (fabs(sm.A[k * kLd + l]) > thresh);
+            big |= (k != l) && (fabs(Ar[k * kLd + l]) > thresh);
         }
         big = __any_sync(0xffffffffu, big);
         if (big && (tid & 31) == 0) sm.flag_rotated = 1;
@@ -318,15 +326,16 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
     }
 
     // ---------------------------------------------------------------- phase 4: sigma, j, d, c
-    if (tid < m) {
-        const double mu = sm.A[tid * kLd + tid];
+    // all M2 positions take part: with odd m the padding index (eigenvalue exactly 0, never retained) may sit anywhere
+    if (tid < M2) {
+        const double mu = Ar[tid * kLd + tid];
         sm.mu[tid] = mu > QN_NOISE_FLOOR * sm.diag_scale ? mu : 0.0;
     }
     asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
-    if (tid < m) {
+    if (tid < M2) {
         const double mine = sm.mu[tid];
         int rank = 0;
-        for (int l = 0; l < m; ++l) {
+        for (int l = 0; l < M2; ++l) {
             const double o = sm.mu[l];
             rank += (o > mine) || (o == mine && l < tid);
         }
@@ -350,16 +359,16 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
     // max_k sigma_k / ||y_k||, with ||y_k||^2 = v_k^T (Theta^T Theta) v_k.
     double tau_use = prm.tau;
     if (prm.tau_cap && prm.partials_theta && prm.source == QN_SRC_PARTIALS && j > 0 && prm.tau > 0.0) {
-        for (int e = tid; e < j * m; e += jthreads) {  // A is free from here on: scratch for the j x m products
+        for (int e = tid; e < j * m; e += jthreads) {  // the copy of A that is not current is free: scratch for the j x m products
             const int k = e / m, a = e % m, col = sm.order[k];
             double bv = 0.0;
-            for (int b = 0; b < m; ++b) bv += sm.B[a * kLd + b] * sm.V[b * kLd + col];
-            sm.A[k * kLd + a] = sm.V[a * kLd + col] * bv;
+            for (int b = 0; b < m; ++b) bv += sm.B[a * kLd + b] * Vr[b * kLd + col];
+            Aw[k * kLd + a] = Vr[a * kLd + col] * bv;
         }
         asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
         if (tid < j) {
             double y2 = 0.0;
-            for (int a = 0; a < m; ++a) y2 += sm.A[tid * kLd + a];
+            for (int a = 0; a < m; ++a) y2 += Aw[tid * kLd + a];
             sm.d[tid] = y2 > 0.0 ? sm.sigma[tid] / sqrt(y2) : 0.0;
         }
         asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
@@ -375,13 +384,13 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
     if (tid < j) {
         const int col = sm.order[tid];
         double dot = 0.0;
-        for (int k = 0; k < m; ++k) dot += sm.V[k * kLd + col] * sm.w[k];
+        for (int k = 0; k < m; ++k) dot += Vr[k * kLd + col] * sm.w[k];
         sm.modec[tid] = dot / sm.mu[col];
     }
     asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
     if (tid < m) {
         double dk = 0.0;
-        for (int r = 0; r < j; ++r) dk += sm.V[tid * kLd + sm.order[r]] * sm.modec[r];
+        for (int r = 0; r < j; ++r) dk += Vr[tid * kLd + sm.order[r]] * sm.modec[r];
         sm.d[tid] = dk;
     }
     asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
