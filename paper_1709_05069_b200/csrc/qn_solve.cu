@@ -23,7 +23,13 @@ struct SolveSmem {
     double A[QN_MAX_M * kLd];
     double V[QN_MAX_M * kLd];  // also scratch for the partial sums before the Jacobi phase
     double A2[QN_MAX_M * kLd], V2[QN_MAX_M * kLd];  // the Jacobi rounds read one copy and write the other
-    double B[QN_MAX_M * kLd];  // reference-shifted Gram of theta (learning-rate cap only)
+    union {
+        double B[QN_MAX_M * kLd];  // reference-shifted Gram of theta (learning-rate cap only; built after the fp32 phase)
+        struct {
+            float A[2][QN_MAX_M * kLd], V[2][QN_MAX_M * kLd];  // fp32 pre-diagonalisation: A / ||A||_F and its rotations
+            float rot_c[QN_MAX_M / 2], rot_s[QN_MAX_M / 2];
+        } f;
+    };
     double w[QN_MAX_M];
     double rowsum[QN_MAX_M];
     double mu[QN_MAX_M];
@@ -51,6 +57,104 @@ __device__ __forceinline__ double block_sum(double x, double* red) {
     double s = 0.0;
     for (int i = 0; i < nw; ++i) s += red[i];
     return s;
+}
+
+// Where physical position i of the tournament table goes after a round: position 0 stays, the other top positions
+// 2k move right, the bottom positions 2k+1 move left, the ends turn round.
+__device__ __forceinline__ int next_pos(int i, int M2) {
+    if (M2 == 2 || i == 0) return i;
+    if (i == 1) return 2;
+    if (i & 1) return i - 2;
+    return i == M2 - 2 ? M2 - 1 : i + 2;
+}
+
+// Pre-diagonalisation in fp32: the same systolic round-robin Jacobi as the fp64 phase of the kernel, on A / ||A||_F.
+// Vector fp64 runs at an eighth of the fp32 rate on this part and bounds the fp64 rounds from m = 32 on; the fp32
+// rounds cost a fraction.  The result is only an approximation (V orthogonal and V^T A V diagonal to about 1e-6):
+// the kernel then re-orthonormalises V in fp64, transforms A with it and lets the fp64 Jacobi finish from there
+// in two or three sweeps.  Returns the buffer index (0 or 1) that holds the final V.
+#ifndef QN_SOLVE_PRE_MIN_M
+#define QN_SOLVE_PRE_MIN_M 12
+#endif
+constexpr int kPreMinM = QN_SOLVE_PRE_MIN_M;  // below this the fp64 sweeps are short anyway
+#ifndef QN_SOLVE_PRE_SWEEPS
+#define QN_SOLVE_PRE_SWEEPS 8
+#endif
+constexpr int kPreMaxSweeps = QN_SOLVE_PRE_SWEEPS;
+__device__ __forceinline__ int jacobi_fp32(SolveSmem& sm, int M2, int tid, int jthreads) {
+    const int H = M2 / 2, N = M2 - 1;
+    const int pa_idx = tid / H, pb_idx = tid % H;
+    const bool worker = tid < H * H;
+    const int ra = 2 * pa_idx, cb = 2 * pb_idx;
+    const int nr0 = next_pos(ra, M2), nr1 = next_pos(ra + 1, M2), nc0 = next_pos(cb, M2), nc1 = next_pos(cb + 1, M2);
+    const float thr_rot = 1e-9f, thr_done = 3e-6f;  // entries are relative to ||A||_F = 1
+    int cur = 0;
+    for (int sweep = 0; sweep < kPreMaxSweeps; ++sweep) {
+        for (int r = 0; r < N; ++r) {
+            const float* Ar = sm.f.A[cur];
+            const float* Vr = sm.f.V[cur];
+            float* Aw = sm.f.A[cur ^ 1];
+            float* Vw = sm.f.V[cur ^ 1];
+            float x00 = 0.f, x01 = 0.f, x10 = 0.f, x11 = 0.f;
+            if (worker) {
+                const float2 r0 = *reinterpret_cast<const float2*>(&Ar[ra * kLd + cb]);
+                const float2 r1 = *reinterpret_cast<const float2*>(&Ar[(ra + 1) * kLd + cb]);
+                x00 = r0.x;
+                x01 = r0.y;
+                x10 = r1.x;
+                x11 = r1.y;
+                if (pa_idx == pb_idx) {
+                    float c = 1.f, sn = 0.f;
+                    if (fabsf(x01) > thr_rot) {
+                        const float df = x11 - x00, of = x01 + x01;
+                        const float r2 = fmaf(df, df, of * of);
+                        const float h = r2 * rsqrtf(r2);
+                        const float tf = copysignf(__fdividef(fabsf(of), fabsf(df) + h), df * of);
+                        c = rsqrtf(fmaf(tf, tf, 1.0f));
+                        sn = tf * c;
+                    }
+                    sm.f.rot_c[pa_idx] = c;
+                    sm.f.rot_s[pa_idx] = sn;
+                }
+            }
+            asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
+            if (worker) {
+                const float ca = sm.f.rot_c[pa_idx], sa = sm.f.rot_s[pa_idx];
+                const float cbr = sm.f.rot_c[pb_idx], sbr = sm.f.rot_s[pb_idx];
+                const float2 v0 = *reinterpret_cast<const float2*>(&Vr[ra * kLd + cb]);
+                const float2 v1 = *reinterpret_cast<const float2*>(&Vr[(ra + 1) * kLd + cb]);
+                const float t00 = cbr * x00 - sbr * x01, t01 = sbr * x00 + cbr * x01;
+                const float t10 = cbr * x10 - sbr * x11, t11 = sbr * x10 + cbr * x11;
+                float y00 = ca * t00 - sa * t10, y10 = sa * t00 + ca * t10;
+                float y01 = ca * t01 - sa * t11, y11 = sa * t01 + ca * t11;
+                if (pa_idx == pb_idx) y01 = y10 = 0.5f * (y01 + y10);
+                Aw[nr0 * kLd + nc0] = y00;
+                Aw[nr0 * kLd + nc1] = y01;
+                Aw[nr1 * kLd + nc0] = y10;
+                Aw[nr1 * kLd + nc1] = y11;
+                Vw[ra * kLd + nc0] = cbr * v0.x - sbr * v0.y;
+                Vw[ra * kLd + nc1] = sbr * v0.x + cbr * v0.y;
+                Vw[(ra + 1) * kLd + nc0] = cbr * v1.x - sbr * v1.y;
+                Vw[(ra + 1) * kLd + nc1] = sbr * v1.x + cbr * v1.y;
+            }
+            asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
+            cur ^= 1;
+        }
+        int big = 0;
+        for (int e = tid; e < M2 * M2; e += jthreads) {
+            const int k = e / M2, l = e % M2;
+            big |= (k != l) && (fabsf(sm.f.A[cur][k * kLd + l]) > thr_done);
+        }
+        big = __any_sync(0xffffffffu, big);
+        if (big && (tid & 31) == 0) sm.flag_rotated = 1;
+        asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
+        const int rotated = sm.flag_rotated;
+        asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
+        if (tid == 0) sm.flag_rotated = 0;
+        asm volatile("bar.sync 1, %0;" ::"r"(jthreads) : "memory");
+        if (!rotated) break;
+    }
+    return cur;
 }
 
 __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
@@ -95,26 +199,6 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
         __syncthreads();
         if (prm.raw_gram)
             for (int e = tid; e < m * m; e += nthr) prm.raw_gram[e] = sm.A[(e / m) * kLd + (e % m)];
-        if (prm.tau_cap && prm.partials_theta) {
-            // the same fixed-order sum for the Gram of theta; it stays reference-shifted: it is only ever applied
-            // to retained v_k, which are orthogonal to the vector of ones, so the centring would change nothing
-            for (int e = tid; e < tri_len; e += nthr) {
-                double s0 = 0, s1 = 0;
-                int p = 0;
-                for (; p + 1 < prm.num_partials_theta; p += 2) {
-                    s0 += prm.partials_theta[(int64_t)(p + 0) * E + e];
-                    s1 += prm.partials_theta[(int64_t)(p + 1) * E + e];
-                }
-                if (p < prm.num_partials_theta) s0 += prm.partials_theta[(int64_t)p * E + e];
-                packed[e] = s0 + s1;
-            }
-            __syncthreads();
-            for (int e = tid; e < m * m; e += nthr) {
-                const int k = e / m, l = e % m;
-                sm.B[k * kLd + l] = packed[k <= l ? qn_tri_index(m, k, l) : qn_tri_index(m, l, k)];
-            }
-            __syncthreads();
-        }
     } else {
         // QN_SRC_WINDOW: the raw Gram (w follows from it in the centring below); QN_SRC_SUMMED: a centred Gram
         // followed by w, e.g. the sum over column shards of what qn_gram wrote (the centring below leaves an
@@ -218,20 +302,95 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
         fro += a * a;
     }
     fro = sqrt(block_sum(fro, sm.red));
+
+    // ---------------------------------------------------------------- phase 3a: fp32 pre-diagonalisation
+    if (m >= kPreMinM && fro > 0.0) {
+        const double scale = 1.0 / fro;
+        for (int e = tid; e < M2 * M2; e += nthr) {
+            const int k = e / M2, l = e % M2;
+            sm.f.A[0][k * kLd + l] = (float)(sm.A[k * kLd + l] * scale);
+            sm.f.V[0][k * kLd + l] = k == l ? 1.f : 0.f;
+        }
+        __syncthreads();
+        int cur = 0;
+        if (tid < jthreads) cur = jacobi_fp32(sm, M2, tid, jthreads);
+        if (tid == 0) sm.j = cur;
+        __syncthreads();
+        cur = sm.j;
+        __syncthreads();
+        // Q = V32 (columns in tournament order) is orthogonal to about 1e-6 only; one Newton-Schulz step
+        // Q <- Q (1.5 I - 0.5 Q^T Q) brings ||Q^T Q - I|| to about 1e-12.  A2 and V2 are free: scratch.
+        for (int e = tid; e < M2 * M2; e += nthr) sm.V[(e / M2) * kLd + (e % M2)] = (double)sm.f.V[cur][(e / M2) * kLd + (e % M2)];
+        __syncthreads();
+        for (int e = tid; e < M2 * M2; e += nthr) {
+            const int i = e / M2, l = e % M2;
+            double acc = 0.0;
+            for (int k = 0; k < M2; ++k) acc = fma(sm.V[k * kLd + i], sm.V[k * kLd + l], acc);
+            sm.A2[i * kLd + l] = (i == l ? 1.5 : 0.0) - 0.5 * acc;
+        }
+        __syncthreads();
+        for (int e = tid; e < M2 * M2; e += nthr) {
+            const int i = e / M2, l = e % M2;
+            double acc = 0.0;
+            for (int k = 0; k < M2; ++k) acc = fma(sm.V[i * kLd + k], sm.A2[k * kLd + l], acc);
+            sm.V2[i * kLd + l] = acc;
+        }
+        __syncthreads();
+        for (int e = tid; e < M2 * M2; e += nthr) sm.V[(e / M2) * kLd + (e % M2)] = sm.V2[(e / M2) * kLd + (e % M2)];
+        __syncthreads();
+        // A <- Q^T A Q (symmetrised): nearly diagonal, in the order of Q's columns; the fp64 Jacobi continues from V = Q
+        for (int e = tid; e < M2 * M2; e += nthr) {
+            const int i = e / M2, l = e % M2;
+            double acc = 0.0;
+            for (int k = 0; k < M2; ++k) acc = fma(sm.A[i * kLd + k], sm.V[k * kLd + l], acc);
+            sm.A2[i * kLd + l] = acc;
+        }
+        __syncthreads();
+        for (int e = tid; e < M2 * M2; e += nthr) {
+            const int i = e / M2, l = e % M2;
+            double acc = 0.0;
+            for (int k = 0; k < M2; ++k) acc = fma(sm.V[k * kLd + i], sm.A2[k * kLd + l], acc);
+            sm.V2[i * kLd + l] = acc;
+        }
+        __syncthreads();
+        for (int e = tid; e < M2 * M2; e += nthr) {
+            const int i = e / M2, l = e % M2;
+            sm.A[i * kLd + l] = 0.5 * (sm.V2[i * kLd + l] + sm.V2[l * kLd + i]);
+        }
+        __syncthreads();
+    }
+    // ---------------------------------------------------------------- phase 1b (learning-rate cap): Gram of theta
+    if (prm.source == QN_SRC_PARTIALS) {
+        const int E = tri_len + m;
+        double* packed = sm.A2;  // free until the fp64 rounds start
+        if (prm.tau_cap && prm.partials_theta) {
+            // the same fixed-order sum for the Gram of theta; it stays reference-shifted: it is only ever applied
+            // to retained v_k, which are orthogonal to the vector of ones, so the centring would change nothing
+            for (int e = tid; e < tri_len; e += nthr) {
+                double s0 = 0, s1 = 0;
+                int p = 0;
+                for (; p + 1 < prm.num_partials_theta; p += 2) {
+                    s0 += prm.partials_theta[(int64_t)(p + 0) * E + e];
+                    s1 += prm.partials_theta[(int64_t)(p + 1) * E + e];
+                }
+                if (p < prm.num_partials_theta) s0 += prm.partials_theta[(int64_t)p * E + e];
+                packed[e] = s0 + s1;
+            }
+            __syncthreads();
+            for (int e = tid; e < m * m; e += nthr) {
+                const int k = e / m, l = e % m;
+                sm.B[k * kLd + l] = packed[k <= l ? qn_tri_index(m, k, l) : qn_tri_index(m, l, k)];
+            }
+            __syncthreads();
+        }
+    }
     if (tid >= jthreads) return;  // the remaining phases synchronise with a named barrier over jthreads
     const double thresh = 1e-15 * fro;
     const double inv_fro = fro > 0.0 ? 1.0 / fro : 0.0;  // brings entries into fp32 range whatever the data's scale
     const int pa_idx = tid / H, pb_idx = tid % H;
     const bool worker = tid < H * H;
-    // where physical position i goes after a round
-    auto next_pos = [&](int i) -> int {
-        if (H == 1 || i == 0) return i;
-        if (i == 1) return 2;
-        if (i & 1) return i - 2;
-        return i == M2 - 2 ? M2 - 1 : i + 2;
-    };
     const int ra = 2 * pa_idx, cb = 2 * pb_idx;  // this thread's block, every round
-    const int nr0 = next_pos(ra), nr1 = next_pos(ra + 1), nc0 = next_pos(cb), nc1 = next_pos(cb + 1);
+    const int nr0 = next_pos(ra, M2), nr1 = next_pos(ra + 1, M2), nc0 = next_pos(cb, M2), nc1 = next_pos(cb + 1, M2);
     double* Ar = sm.A;
     double* Aw = sm.A2;
     double* Vr = sm.V;
