@@ -35,7 +35,7 @@ def _rank_main(rank, world, port, out):
 
 def test_two_replicas_report_the_slowest_rank_and_the_whole_job():
     world, port = 2, _free_port()
-    with mp.Manager() as mgr:
+    with mp.get_context("spawn").Manager() as mgr:
         out = mgr.dict()
         mp.spawn(_rank_main, args=(world, port, out), nprocs=world, join=True)
         res = dict(out)
@@ -107,7 +107,7 @@ def test_sharded_gram_buffers_add_up_to_the_whole_problem():
     import workloads as W
 
     world, port = 2, _free_port()
-    with mp.Manager() as mgr:
+    with mp.get_context("spawn").Manager() as mgr:
         out = mgr.dict()
         mp.spawn(_shard_rank_main, args=(world, port, out), nprocs=world, join=True)
         res = dict(out)
