@@ -144,13 +144,16 @@ __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
 
 // One work item = kPairs pairs of columns of every row: a 16-byte vector for fp32 storage (4 columns), HALF a vector for
 // bf16 storage (8 bytes, 4 columns).  With whole bf16 vectors the per-thread state (five packed quantities per pair and
-// the loads in flight) takes 108 registers, two CTAs fit an SM and the pass is latency-bound at 5.8 TB/s; with half
-// vectors and eight Workers in flight it takes about 60 and four CTAs fit.
+// the loads in flight) takes 108 registers, two CTAs of 256 fit an SM and the pass is latency-bound at 5.8 TB/s.  With
+// half vectors, four Workers (eight loads) in flight and CTAs of 128 threads it takes 56 registers and nine CTAs fit:
+// measured 6.5 TB/s at m = 8, 6.7 at m = 16, 7.0 at m = 64 (eight Workers in flight, 78 registers, CTAs of 256: 6.1,
+// 6.5, 6.9; two Workers in flight: 5.3, 5.6, 6.0).  fp32 storage: 6.95 TB/s at m = 32 either way.
 template <typename T>
 struct CombineItem {
     static constexpr int kPairs = 2;
     static constexpr int kCols = 4;
-    static constexpr int kUnroll = sizeof(T) == 2 ? 8 : 4;  // Workers whose loads are in flight together
+    static constexpr int kThreads = sizeof(T) == 2 ? 128 : kCombineThreads;
+    static constexpr int kUnroll = 4;  // Workers whose loads are in flight together
     // pair p (0 or 1) of the item as two floats
     static __device__ __forceinline__ f32x2 pair(const uint2& lo, const uint2& hi, int p);
 };
@@ -175,18 +178,17 @@ __device__ __forceinline__ void load_item(const T* p, uint2& lo, uint2& hi) {
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kCombineThreads)
+__global__ void __launch_bounds__(CombineItem<T>::kThreads)
 combine_vec_kernel(const T* __restrict__ theta, const T* __restrict__ g, int64_t n, int m,
                    const qn_coef_block* __restrict__ coef, T* __restrict__ out, const T* __restrict__ base) {
     using Item = CombineItem<T>;
-    constexpr int kCols = Item::kCols, kPairs = Item::kPairs, kUnroll = Item::kUnroll;
+    constexpr int kCols = Item::kCols, kPairs = Item::kPairs, kUnroll = Item::kUnroll, kThreads = Item::kThreads;
     __shared__ float c_sh[QN_MAX_M];
-    if (threadIdx.x < QN_MAX_M) c_sh[threadIdx.x] = coef->c[threadIdx.x];
+    for (int k = threadIdx.x; k < QN_MAX_M; k += kThreads) c_sh[k] = coef->c[k];
     const float tau = coef->tau, inv_m = coef->inv_m;
     __syncthreads();
     const int64_t nitems = n / kCols;
-    for (int64_t item = (int64_t)blockIdx.x * kCombineThreads + threadIdx.x; item < nitems;
-         item += (int64_t)gridDim.x * kCombineThreads) {
+    for (int64_t item = (int64_t)blockIdx.x * kThreads + threadIdx.x; item < nitems; item += (int64_t)gridDim.x * kThreads) {
         const int64_t i0 = item * kCols;
         f32x2 th0[kPairs], g0[kPairs], sth[kPairs], sg[kPairs], acc[kPairs];
         {
@@ -252,19 +254,21 @@ static cudaError_t launch_combine_t(const T* theta, const T* g, int64_t n, int m
     const bool aligned = (reinterpret_cast<uintptr_t>(theta) % 16 == 0) && (reinterpret_cast<uintptr_t>(g) % 16 == 0) &&
                          (reinterpret_cast<uintptr_t>(out) % 16 == 0) && (reinterpret_cast<uintptr_t>(base) % 16 == 0) &&
                          ((n * (int64_t)sizeof(T)) % 16 == 0);
+    const int threads = aligned ? CombineItem<T>::kThreads : kCombineThreads;
     const int64_t nitems = aligned ? n / CombineItem<T>::kCols : n;
-    const int64_t want = (nitems + kCombineThreads - 1) / kCombineThreads;
+    const int64_t want = (nitems + threads - 1) / threads;
     int per_sm = 1;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, combine_vec_kernel<T>, kCombineThreads, 0) != cudaSuccess ||
-        per_sm < 1)
-        per_sm = 1;
+    const cudaError_t oe =
+        aligned ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, combine_vec_kernel<T>, threads, 0)
+                : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, combine_kernel<T, false>, threads, 0);
+    if (oe != cudaSuccess || per_sm < 1) per_sm = 1;
     // whole waves only: a grid-strided loop gains nothing from a partial last wave
-    const int64_t cap = (int64_t)qn_sm_count() * per_sm * 2;
+    const int64_t cap = (int64_t)qn_sm_count() * per_sm * 4;
     const int grid = (int)(want < cap ? (want > 0 ? want : 1) : cap);
     if (aligned)
-        combine_vec_kernel<T><<<grid, kCombineThreads, 0, st>>>(theta, g, n, m, coef, out, base);
+        combine_vec_kernel<T><<<grid, threads, 0, st>>>(theta, g, n, m, coef, out, base);
     else
-        combine_kernel<T, false><<<grid, kCombineThreads, 0, st>>>(theta, g, n, m, coef, out, base);
+        combine_kernel<T, false><<<grid, threads, 0, st>>>(theta, g, n, m, coef, out, base);
     return cudaGetLastError();
 }
 

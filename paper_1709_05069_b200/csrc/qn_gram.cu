@@ -7,7 +7,9 @@
 // Arithmetic, three modes:
 //   kFast     fp32 products, fp32 accumulation over at most kFlushCols columns per thread, then fp64.
 //             The rounding errors of the products are unbiased and average out as 1/sqrt(n); used
-//             for n >= QN_PRECISE_BELOW, where they stay below 1e-10 of the largest eigenvalue.
+//             for n >= QN_PRECISE_BELOW, where they stay below 1e-10 of the largest eigenvalue.  (Measured with
+//             this mode forced at n = 2^20, m = 16 and a spectrum that reaches down to lambda = 1e-3: sigma error
+//             0.9 of the 1e-5 bar against 0.001 in kPrecise, and the pass is no faster there.)
 //   kPrecise  the shifted values are rounded to fp32 once, every product and sum is fp64 (a product of
 //             two fp32 values is exact in fp64), so the result is the exact Gram of slightly perturbed
 //             data and stays positive semi-definite to fp64 accuracy; used for small n.
@@ -256,6 +258,11 @@ constexpr int kGsWarps = 7;                   // warps that do the arithmetic; o
 constexpr int kGsThreads = (kGsWarps + 1) * 32;  // so that every thread can have the registers its 132 sums need
 constexpr int kGsSeg = kGsWarps * 32 * 16;    // bytes of one row in a stage: one 16-byte vector per arithmetic thread
 constexpr int kGsStages = 7;
+// Columns that one half of a packed fp32 accumulator sums between flushes to fp64.  The flush costs fp64-pipe time
+// (bf16 storage, m = 8: 4.40 TB/s with 32 columns, 4.62 with 64, 4.85 with 512); the measured sigma error on inputs
+// with a spectral gap is 0.035 of the 1e-5 bar with 64 columns at n = 2^22 and 2^24 alike (0.015 with 32; with 128
+// it grows with n).
+constexpr int kGsFlushCols = 64;
 static_assert(kGsThreads == kThreads, "the reduction of the direct kernels is written for kThreads threads");
 
 struct GsSmem {
@@ -275,8 +282,8 @@ gram_stream_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict
     constexpr int kSegCols = kGsSeg / (int)sizeof(T);   // columns of one row segment
     constexpr int NB = kDirectM / MR;                    // a stage's 8 segments hold NB column blocks of MR rows, so that
     constexpr int kTileCols = NB * kSegCols;             // every m keeps the same number of bytes in flight
-    // each half of a packed accumulator sums every other column: kFlushCols columns per half between flushes
-    constexpr int kFlushIters = 2 * kFlushCols / kCols;
+    // each half of a packed accumulator sums every other column: kGsFlushCols columns per half between flushes
+    constexpr int kFlushIters = 2 * kGsFlushCols / kCols;
     constexpr uint64_t kUsed = gs_used_mask(MR);  // the sums this instance forms
     extern __shared__ unsigned char smem_raw[];
     GsSmem& sm = *reinterpret_cast<GsSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
