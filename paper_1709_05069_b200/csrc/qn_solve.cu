@@ -81,13 +81,19 @@ constexpr int kPreMinM = QN_SOLVE_PRE_MIN_M;  // below this the fp64 sweeps are 
 #define QN_SOLVE_PRE_SWEEPS 8
 #endif
 constexpr int kPreMaxSweeps = QN_SOLVE_PRE_SWEEPS;
+// largest off-diagonal entry (relative to ||A||_F) at which the fp32 sweeps stop.  Measured totals of the kernel in
+// thousands of cycles at m = 16 / 32 / 64: 3e-6: 164 / 330 / 1287, 3e-5: 163 / 335 / 1343, 3e-4: 152 / 354 / 1414,
+// 3e-3: 159 / 374 / 1621 (a looser stop saves fp32 sweeps and costs more fp64 sweeps, which are 1.6 times as long).
+#ifndef QN_SOLVE_PRE_THR
+#define QN_SOLVE_PRE_THR 3e-6f
+#endif
 __device__ __forceinline__ int jacobi_fp32(SolveSmem& sm, int M2, int tid, int jthreads) {
     const int H = M2 / 2, N = M2 - 1;
     const int pa_idx = tid / H, pb_idx = tid % H;
     const bool worker = tid < H * H;
     const int ra = 2 * pa_idx, cb = 2 * pb_idx;
     const int nr0 = next_pos(ra, M2), nr1 = next_pos(ra + 1, M2), nc0 = next_pos(cb, M2), nc1 = next_pos(cb + 1, M2);
-    const float thr_rot = 1e-9f, thr_done = 3e-6f;  // entries are relative to ||A||_F = 1
+    const float thr_rot = 1e-9f, thr_done = QN_SOLVE_PRE_THR;  // entries are relative to ||A||_F = 1
     int cur = 0;
     for (int sweep = 0; sweep < kPreMaxSweeps; ++sweep) {
         for (int r = 0; r < N; ++r) {
