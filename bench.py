@@ -17,6 +17,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import sys
 import threading
@@ -154,18 +155,31 @@ def dist_env():
     return rank, world, local
 
 
-def oracle_sample_time(cfg: W.Config, lam: float, target_cols: int):
-    """Time the CPU oracle, as it stands, on the first `target_cols` columns of the workload."""
-    import oracle
+class OracleSample:
+    """The first `target_cols` columns of the workload on the host, and the CPU oracle, as it stands, timed on them."""
 
-    sub = cfg.with_shape(n=min(cfg.n, target_cols))
-    theta, g = W.generate(sub, "cpu")
-    tb, gb = W.to_bits(theta), W.to_bits(g)
-    cores = oracle.threads_used(0)
-    t0 = time.perf_counter()
-    oracle.update(tb, gb, cfg.tau, lam)
-    dt = time.perf_counter() - t0
-    return dt, sub.n, cores
+    def __init__(self, cfg: W.Config, target_cols: int):
+        import oracle
+
+        self.oracle = oracle
+        self.cfg = cfg
+        sub = cfg.with_shape(n=min(cfg.n, target_cols))
+        theta, g = W.generate(sub, "cpu")
+        self.tb, self.gb = W.to_bits(theta), W.to_bits(g)
+        self.ncols = sub.n
+        self.cores = oracle.threads_used(0)
+
+    def time_once(self) -> float:
+        t0 = time.perf_counter()
+        self.oracle.update(self.tb, self.gb, self.cfg.tau, self.cfg.lam)
+        return time.perf_counter() - t0
+
+    def time_for(self, seconds: float, max_reps: int = 64):
+        """Mean time of one oracle update over enough repetitions to fill about `seconds` of CPU work."""
+        first = self.time_once()
+        reps = max(1, min(max_reps, int(math.ceil(seconds / max(first, 1e-3))) - 1))
+        times = [self.time_once() for _ in range(reps)]
+        return float(np.mean(times)), reps
 
 
 def run_reference(args, cfg: W.Config):
@@ -175,11 +189,11 @@ def run_reference(args, cfg: W.Config):
     import oracle
 
     oracle.build()
-    sample_cols = min(cfg.n, args.ref_cols)
+    sample = OracleSample(cfg, args.ref_cols)
+    ncols, cores = sample.ncols, sample.cores
     times = []
-    cores = None
     for it in range(args.warmup + args.steps):
-        dt, ncols, cores = oracle_sample_time(cfg, cfg.lam, sample_cols)
+        dt = sample.time_once()
         if it >= args.warmup:
             times.append(dt)
     per_update = float(np.mean(times)) * (cfg.n / ncols)
@@ -217,6 +231,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--ref-cols", type=int, default=6_400_000, help="columns per oracle sample")
+    ap.add_argument("--ref-seconds", type=float, default=12.0, help="CPU work of the cpu_baseline leg, seconds")
     args = ap.parse_args()
 
     cfg = W.CONFIGS[args.config].with_shape(n=args.n, m=args.m)
@@ -256,11 +271,13 @@ def main():
         import oracle
 
         oracle.build()
-        dt, ncols, cores = oracle_sample_time(cfg, cfg.lam, args.ref_cols)
-        per_update = dt * (cfg.n / ncols)
-        cpu_baseline = {"value": 1.0 / per_update, "unit": UNIT, "cores": cores, "kind": "oracle",
-                        "sample": "one oracle update on the first %d of %d columns (%.1f s), time scaled by n/sample"
-                                  % (ncols, cfg.n, dt)}
+        sample = OracleSample(cfg, args.ref_cols)
+        dt, reps = sample.time_for(args.ref_seconds)
+        per_update = dt * (cfg.n / sample.ncols)
+        cpu_baseline = {"value": 1.0 / per_update, "unit": UNIT, "cores": sample.cores, "kind": "oracle",
+                        "sample": "%d oracle updates on the first %d of %d columns (%.1f s of CPU work after one warm-up "
+                                  "update), mean time scaled by n/sample" % (reps, sample.ncols, cfg.n, dt * reps)}
+        del sample
 
     # ------------------------------------------------------------------ inputs resident in HBM
     theta, g = W.generate(cfg, dev)
