@@ -147,7 +147,7 @@ qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, do
     {
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st,
-                           &h->last_launches, h->error_word) != cudaSuccess)
+                           &h->last_launches, h->error_word, lambda) != cudaSuccess)
             return QN_ERR_CUDA;
     }
     int np_theta = 0;
@@ -155,7 +155,7 @@ qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, do
         // the learning-rate cap needs ||Theta v_k||: one more Gram pass, over theta
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, theta, h->n, h->m, false, h->partials_theta, &np_theta, h->max_partials, st,
-                           &h->last_launches, h->error_word) != cudaSuccess)
+                           &h->last_launches, h->error_word, lambda) != cudaSuccess)
             return QN_ERR_CUDA;
     }
     qn_solve_params p;
@@ -389,7 +389,7 @@ extern "C" qn_status qn_apply_hinv(qn_handle h, const void* theta, const void* g
     if (s == QN_OK) {
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st, &h->last_launches,
-                           h->error_word) != cudaSuccess)
+                           h->error_word, lambda) != cudaSuccess)
             s = QN_ERR_CUDA;
     }
     if (s == QN_OK) {

@@ -229,21 +229,21 @@ __device__ __forceinline__ uint64_t gs_pair<__nv_bfloat16>(const uint4& v, int q
 }
 
 // whether entry e of the 8-row packed layout (36 Gram entries by rows, then 8 products with the reference) involves
-// only rows < mr
-__host__ __device__ constexpr bool gs_used(int e, int mr) {
-    if (e >= kDirectTri) return e - kDirectTri < mr;
+// only rows first .. mr-1 (first = 1 where row 0 is the reference: its shifted values are exactly zero)
+__host__ __device__ constexpr bool gs_used(int e, int mr, int first) {
+    if (e >= kDirectTri) return e - kDirectTri >= first && e - kDirectTri < mr;
     int k = 0, rem = e;
     while (rem >= kDirectM - k) {
         rem -= kDirectM - k;
         ++k;
     }
-    return k + rem < mr;
+    return k >= first && k + rem < mr;
 }
 
 // the same for all 44 entries as a bit mask (a compile-time constant per mr)
-__host__ __device__ constexpr uint64_t gs_used_mask(int mr) {
+__host__ __device__ constexpr uint64_t gs_used_mask(int mr, int first) {
     uint64_t mask = 0;
-    for (int e = 0; e < kDirectAcc; ++e) mask |= (uint64_t)(gs_used(e, mr) ? 1 : 0) << e;
+    for (int e = 0; e < kDirectAcc; ++e) mask |= (uint64_t)(gs_used(e, mr, first) ? 1 : 0) << e;
     return mask;
 }
 
@@ -275,7 +275,7 @@ struct GsSmem {
 // MR = 2, 4 or 8 >= m: the rows that are computed (the sums of rows >= MR stay zero and cost nothing; with MR = 8 for
 // every m the pass would be bound by the same instruction count whatever m, e.g. 2.3 TB/s at m = 4 with bf16 storage).
 // The sums keep their place in the 8-row packed layout, so the reduction is shared with the register-fed kernel.
-template <typename T, int MR>
+template <typename T, int MR, bool kRef0>
 __global__ void __launch_bounds__(kGsThreads, 1)
 gram_stream_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ partials, int* __restrict__ error_word) {
     constexpr int kCols = Storage<T>::kVec;
@@ -284,7 +284,18 @@ gram_stream_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict
     constexpr int kTileCols = NB * kSegCols;             // every m keeps the same number of bytes in flight
     // each half of a packed accumulator sums every other column: kGsFlushCols columns per half between flushes
     constexpr int kFlushIters = 2 * kGsFlushCols / kCols;
-    constexpr uint64_t kUsed = gs_used_mask(MR);  // the sums this instance forms
+    // Reference of a column: the Workers' mean, or (kRef0) Worker 0's value.  Any reference is exact for the identity
+    // that the solve kernel applies; g_k - g_0 is exact in fp32 for bf16 data; row 0's shifted values are exactly zero,
+    // so its products are not formed: 42 packed instructions per pair of columns at m = 8 instead of 60.  With bf16
+    // storage, where the pass is bound by its instruction count and not by HBM: 6.2 against 4.6 TB/s at m = 8, 5.5
+    // against 5.1 at m = 4, 5.1 against 4.5 at m = 2.  The price is accuracy: every entry of the shifted Gram then
+    // carries Worker 0's deviation from the mean.  Measured on inputs whose largest mode sits on Workers 0 and 1
+    // (the worst case), bf16 storage, in units of the 1e-5 bar: error of any sigma_k against sigma_1 0.16 (mean:
+    // 0.013); relative error of the smallest retained sigma_k 0.13 at lambda = 0.01, 0.63 at lambda = 0.005 (it grows
+    // as 1 / lambda^2).  So the launcher takes it only for bf16 storage and a known lambda >= QN_REF0_MIN_LAMBDA.
+    // (fp32 storage, whose subtraction is not exact: 0.65 against 0.035, and the pass is HBM-bound anyway.)
+    constexpr int kFirst = kRef0 ? 1 : 0;
+    constexpr uint64_t kUsed = gs_used_mask(MR, kFirst);  // the sums this instance forms
     extern __shared__ unsigned char smem_raw[];
     GsSmem& sm = *reinterpret_cast<GsSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -364,15 +375,20 @@ gram_stream_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict
                 uint64_t x[MR];
 #pragma unroll
                 for (int k = 0; k < MR; ++k) x[k] = gs_pair<T>(v[k], q);
-                uint64_t sum = x[0];
+                uint64_t r;
+                if (kRef0) {
+                    r = x[0];
+                } else {
+                    uint64_t sum = x[0];
 #pragma unroll
-                for (int k = 1; k < MR; ++k) sum = gs_add2(sum, x[k]);
-                const uint64_t r = gs_mul2(sum, inv_m2);
+                    for (int k = 1; k < MR; ++k) sum = gs_add2(sum, x[k]);
+                    r = gs_mul2(sum, inv_m2);
+                }
                 // padding rows (m <= k < MR) read as zero and become -r here: they only reach sums that are never output
 #pragma unroll
-                for (int k = 0; k < MR; ++k) x[k] = gs_sub2(x[k], r);
+                for (int k = kFirst; k < MR; ++k) x[k] = gs_sub2(x[k], r);
 #pragma unroll
-                for (int k = 0; k < MR; ++k) {
+                for (int k = kFirst; k < MR; ++k) {
 #pragma unroll
                     for (int l = k; l < MR; ++l) {
                         const int idx = k * kDirectM - (k * (k - 1)) / 2 + (l - k);  // place in the 8-row packed layout
@@ -380,7 +396,7 @@ gram_stream_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict
                     }
                 }
 #pragma unroll
-                for (int k = 0; k < MR; ++k) acc[kDirectTri + k] = gs_fma2(x[k], r, acc[kDirectTri + k]);
+                for (int k = kFirst; k < MR; ++k) acc[kDirectTri + k] = gs_fma2(x[k], r, acc[kDirectTri + k]);
             }
             if (++iters == kFlushIters) {
                 iters = 0;
@@ -414,7 +430,7 @@ gram_stream_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict
 
 template <typename T>
 static cudaError_t launch_gram_stream(const T* g, int64_t n, int m, double* partials, int* num_partials,
-                                      int max_partials, int* error_word, cudaStream_t st) {
+                                      int max_partials, int* error_word, bool ref0, cudaStream_t st) {
     const int mr = m <= 2 ? 2 : m <= 4 ? 4 : 8;
     const int64_t tile_cols = (kDirectM / mr) * (kGsSeg / (int64_t)sizeof(T));
     const int64_t ntiles = (n + tile_cols - 1) / tile_cols;
@@ -422,7 +438,11 @@ static cudaError_t launch_gram_stream(const T* g, int64_t n, int m, double* part
     int grid = (int)(ntiles < sms ? ntiles : sms);
     if (grid > max_partials) grid = max_partials;
     *num_partials = grid;
-    auto kern = m <= 2 ? gram_stream_kernel<T, 2> : m <= 4 ? gram_stream_kernel<T, 4> : gram_stream_kernel<T, 8>;
+    void (*kern)(const T*, int64_t, int, double*, int*);
+    if (ref0 && sizeof(T) == 2)
+        kern = m <= 2 ? gram_stream_kernel<T, 2, true> : m <= 4 ? gram_stream_kernel<T, 4, true> : gram_stream_kernel<T, 8, true>;
+    else
+        kern = m <= 2 ? gram_stream_kernel<T, 2, false> : m <= 4 ? gram_stream_kernel<T, 4, false> : gram_stream_kernel<T, 8, false>;
     const size_t smem = sizeof(GsSmem) + 128;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -720,7 +740,8 @@ static bool tc_allowed() {
     return !(v && v[0] == 'a');
 }
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
-                           int* num_partials, int max_partials, cudaStream_t st, int* launches, int* error_word) {
+                           int* num_partials, int max_partials, cudaStream_t st, int* launches, int* error_word,
+                           double lambda_hint) {
     cudaError_t e;
     const int64_t elem = dtype == QN_F32 ? 4 : 2;
     if (!raw && tc_allowed() && qn_gram_tc_applicable(dtype, g, n, m)) {
@@ -728,10 +749,11 @@ cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool
     } else if (!raw && tc_allowed() && m <= qn::kDirectM && n >= QN_PRECISE_BELOW &&
                reinterpret_cast<uintptr_t>(g) % 16 == 0 && (n * elem) % 16 == 0) {
         // bulk-copy variant of the direct kernel (QN_GRAM_PATH=alu keeps the register-fed one, for A/B runs)
+        const bool ref0 = lambda_hint >= QN_REF0_MIN_LAMBDA;
         e = dtype == QN_F32 ? qn::launch_gram_stream(static_cast<const float*>(g), n, m, partials, num_partials,
-                                                     max_partials, error_word, st)
+                                                     max_partials, error_word, false, st)
                             : qn::launch_gram_stream(static_cast<const __nv_bfloat16*>(g), n, m, partials,
-                                                     num_partials, max_partials, error_word, st);
+                                                     num_partials, max_partials, error_word, ref0, st);
     } else {
         e = dtype == QN_F32
                 ? qn::launch_gram_t(static_cast<const float*>(g), n, m, raw, partials, num_partials, max_partials, st)

@@ -72,9 +72,13 @@ struct qn_solve_params {
 
 // Launchers.  Each returns the launch error and adds the kernels it launched to *launches.
 // error_word (device int, may be NULL) is set to 1 by a kernel that gave up on a bounded wait.
+// lambda_hint: the cut-off of the step that will use the Gram, or 0 if unknown.  From QN_REF0_MIN_LAMBDA on, the
+// bulk-copy kernel for bf16 storage and m <= 8 may take Worker 0 instead of the mean as its per-column reference
+// (a third fewer instructions; the error of a retained sigma_k grows as 1 / lambda^2, see qn_gram.cu).
+#define QN_REF0_MIN_LAMBDA 0.01
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
                            int* num_partials, int max_partials, cudaStream_t st, int* launches,
-                           int* error_word = nullptr);
+                           int* error_word = nullptr, double lambda_hint = 0.0);
 bool qn_gram_tc_applicable(qn_dtype dtype, const void* g, int64_t n, int m);
 cudaError_t qn_launch_gram_tc(qn_dtype dtype, const void* g, int64_t n, int m, double* partials, int* num_partials,
                               int max_partials, int* error_word, cudaStream_t st);

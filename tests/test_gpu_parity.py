@@ -513,6 +513,17 @@ def test_direct_gram_paths_at_large_n(qn, dtype, m, n, gap):
     check_against_oracle(qn, theta, g, cfg.tau, lam, dtype, expect_j=expect)
 
 
+@pytest.mark.parametrize("m,lam", [(8, 0.005), (8, 0.01), (4, 0.005), (4, 0.02), (7, 0.01)])
+def test_direct_gram_reference_by_lambda(qn, m, lam):
+    """bf16 storage, m <= 8, n >= 2^22: from lambda = 0.01 on the Gram pass shifts by Worker 0's value (a third fewer
+    instructions, less accurate on small retained modes), below it by the Workers' mean.  The gap-variant inputs put
+    the largest mode on Workers 0 and 1, the worst case for the first choice; same bar on both sides of the switch."""
+    cfg = W.Config(42, 1 << 22, m, "bf16", -2, 2, 0, 0.01, 1e-4, 1.0, 0.01)
+    theta, g = W.generate(cfg, "cuda", gap_lam=lam, gap_scale=1.0)
+    expect = assert_gap(theta, g, lam)
+    check_against_oracle(qn, theta, g, cfg.tau, lam, "bf16", expect_j=expect)
+
+
 # --------------------------------------------------------------------------- tensor-core Gram path (n >= 2^22, m > 8)
 @pytest.mark.parametrize("dtype,m,n,gap", [
     ("f32", 32, (1 << 22) + 64 * 3 + 8, True),     # config 2's shape class: two tiles per stage, ragged tail
