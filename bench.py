@@ -58,7 +58,7 @@ MEASURED_TRAFFIC_RATIO = {
     ("row", "bf16", "direct"): 0.979,  # row_stream_kernel<bf16>, config 3's generator at n = 33,554,432
     ("combine", "bf16", "direct"): 0.986,  # combine_vec_kernel<bf16>, config 4's generator at m = 8, n = 33,554,432
     ("combine", "bf16", "tc"): 0.986,      # the same kernel (the Gram path does not change the combine pass)
-    ("gram", "bf16", "direct"): 1.007,     # gram_stream_kernel<bf16, 8>, same capture
+    ("gram", "bf16", "direct"): 1.008,     # gram_stream_kernel<bf16, 8, true>, same capture
 }
 
 
