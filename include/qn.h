@@ -93,6 +93,11 @@ QN_API qn_status qn_destroy(qn_handle h);
  *   j_out        HOST int32, may be NULL
  *   sigma_out    HOST double[m], descending, may be NULL
  * If both j_out and sigma_out are NULL the call does not wait for the device.
+ * Accuracy against the exact fp64 evaluation of Eq. (2)-(4) on the stored values: j exact when no sigma_k
+ * lies within 1e-5 sigma_1 of lambda sigma_1; every sigma_k within 1e-5 sigma_1, the retained ones within a
+ * relative 1e-5; theta_new within a relative L2 error of 1e-5 (fp32 storage) or 2e-3 (bf16 storage: the single
+ * rounding of the output).  The arithmetic of the Gram pass is chosen from n, m, the storage type and lambda
+ * (fp64 products below 2^22 parameters; fp32 or tensor-core products above), never from the data.
  */
 QN_API qn_status qn_update(qn_handle h, const void* theta, const void* g, double tau, double lambda,
                     void* theta_new, int32_t* j_out, double* sigma_out, void* cuda_stream);
