@@ -428,3 +428,27 @@ def test_quadratic_convergence_direction():
     B, _ = np.linalg.qr(np.concatenate([U, Y], axis=1))
     resid = diff - B @ (B.T @ diff)
     assert np.linalg.norm(resid) <= 1e-9 * np.linalg.norm(diff)
+
+
+def test_stored_small_cases_still_hold(oracle_mod):
+    """Regression anchor: the oracle's results on formula-given inputs, as written by tests/golden/make_golden.py.
+    (Not a pin: the values came from the oracle.  It makes a change of the oracle's arithmetic visible.)"""
+    import importlib.util
+    import json
+    import os
+
+    here = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    spec = importlib.util.spec_from_file_location("make_golden", os.path.join(here, "make_golden.py"))
+    mg = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mg)
+    with open(os.path.join(here, "oracle_small_cases.json")) as f:
+        cases = json.load(f)["cases"]
+    assert [(c["m"], c["n"], c["tau"], c["lam"]) for c in cases] == mg.CASES
+    for c in cases:
+        theta, g = mg.inputs(c["m"], c["n"])
+        r = oracle_mod.update(theta, g, c["tau"], c["lam"])
+        assert r.j == c["j"]
+        sigma = np.array([float.fromhex(x) for x in c["sigma"]])
+        want = np.array([float.fromhex(x) for x in c["theta_new"]])
+        assert np.max(np.abs(r.sigma - sigma)) <= 1e-12 * sigma[0]
+        assert np.max(np.abs(r.theta_new - want)) <= 1e-10 * np.max(np.abs(want))
