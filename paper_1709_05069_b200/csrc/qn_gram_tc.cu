@@ -58,9 +58,31 @@
 
 namespace qn {
 
-constexpr int kTcProducers = 10;
 constexpr int kTcMmaWarps = 2;
-constexpr int kTcThreads = (4 + kTcMmaWarps + kTcProducers) * 32;
+#ifndef QN_TC_PRODUCERS_BF16
+#define QN_TC_PRODUCERS_BF16 10
+#endif
+#ifndef QN_TC_PRODUCERS_64
+#define QN_TC_PRODUCERS_64 8
+#endif
+// Warp roles.  Warps 4-7 drain (a warp reads the TMEM lanes of quadrant warp % 4), two warps issue the MMAs, the rest
+// convert.  A warp's scheduler is warp % 4.  16 warps, ten producers (3, 2, 3, 2 per scheduler), except bf16 storage
+// at MP = 64: the ring holds eight stages, i.e. the items of four teams of two warps, so a fifth team mostly waits for a
+// stage, and the conversion is bound by the schedulers' issue rate: 14 warps, eight producers, two on every scheduler
+// (measured 3.65 against 3.56 TB/s; registers are allocated to warps in fours, so 14 warps get no more than 16 would).
+// fp32 storage at MP = 64 waits for its loads instead and needs the ten warps' bytes in flight (4.4 against 3.7 TB/s).
+template <typename T, int MP>
+struct TcRoles {
+    static constexpr int kProducers = sizeof(T) == 2 ? (MP == 64 ? QN_TC_PRODUCERS_64 : QN_TC_PRODUCERS_BF16) : 10;
+    static constexpr bool kEight = kProducers == 8;
+    static constexpr int kThreads = (4 + kTcMmaWarps + kProducers) * 32;
+    static constexpr int kMmaWarp = kEight ? 12 : 3, kMmaWarpB = kEight ? 13 : 9, kDrainWarp0 = 4;
+    // producer index 0 .. kProducers-1 of a warp that neither drains nor issues
+    static __device__ __forceinline__ int producer_index(int warp) {
+        if (kEight) return warp < 4 ? warp : warp - 4;                    // warps 0-3, 8-11
+        return warp < 3 ? warp : warp == 8 ? 3 : warp - 6;                // warps 0-2, 8, 10-15
+    }
+};
 constexpr int kTcStageRows = 144;                 // 128 operand rows + 16 rows for the references (B operand only)
 constexpr int kTcStageBytes = kTcStageRows * 128;
 constexpr int kTcRelease = 2;                     // stages released to the producers by one commit
@@ -93,7 +115,7 @@ struct TcShape {
     static constexpr int kRowGroups = kRowsPerWarp / kRowsPerLane;      // lanes of a warp that share a column chunk
     static constexpr int kChunksPerItem = 32 / kRowGroups;              // 8-column chunks of one work item
     static constexpr int kTeam = MP / kRowsPerWarp;                     // warps that share the columns of an item
-    static constexpr int kTeams = kTcProducers / kTeam;
+    static constexpr int kTeams = TcRoles<T, MP>::kProducers / kTeam;
     static constexpr int kItemCols = 8 * kChunksPerItem;
     static constexpr int kTilesPerStage = 64 / MP;
     static constexpr int kStageCols = 64 * kTilesPerStage;
@@ -104,7 +126,7 @@ struct TcShape {
     static constexpr int kStageRowBytes = kStageCols * (int)sizeof(T);
     static constexpr int kRun = kStageRowBytes >= kTcRunBytes ? 1 : kTcRunBytes / kStageRowBytes;
     static constexpr int kStages = MP == 64 ? 8 : 10;
-    static_assert(kRowGroups >= 1 && kTcProducers % kTeam == 0 && kRun % kStagesPerItem == 0, "shape");
+    static_assert(kRowGroups >= 1 && TcRoles<T, MP>::kProducers % kTeam == 0 && kRun % kStagesPerItem == 0, "shape");
     static_assert(kStagesPerItem <= kTcRelease, "the stages of an item belong to one release group");
     // Stages per accumulation chain = per drain.  The error of a chain grows with its length; bf16 storage
     // (hi + lo exact, no input rounding at all) has the margin for 16 instructions, fp32 storage keeps 8.
@@ -126,7 +148,7 @@ struct TcSmem {
     uint32_t tmem_base;
     int abort;
     // column sums exchanged by the two warps of a team (MP = 64): [team][item parity][warp of the team][chunk]
-    alignas(16) uint4 xbuf[MP == 64 ? kTcProducers / 2 : 1][2][2][16][2];
+    alignas(16) uint4 xbuf[MP == 64 ? 5 : 1][2][2][16][2];
 };
 
 // K-major, 128-byte swizzle, 8-row groups 1024 bytes apart (the stage built by the producer warps).
@@ -219,7 +241,7 @@ __device__ __forceinline__ void st_shared16_if(const void* p, const uint32_t (&v
 
 // kFull: m == MP, every operand row belongs to a Worker (the row loops then run without branches).
 template <typename T, int MP, bool kFull>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(TcRoles<T, MP>::kThreads, 1)
 gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ partials, int* __restrict__ error_word) {
     using Shape = TcShape<T, MP>;
     using Smem = TcSmem<MP>;
@@ -238,7 +260,9 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
     volatile int* abort = &sm.abort;
     // Roles by warp: 3 and 9 = MMA issue (on different schedulers), 4..7 = drain (TMEM quadrant = warp - 4 =
     // warp % 4), the rest = producers.
-    constexpr int kMmaWarp = 3, kMmaWarpB = 9, kDrainWarp0 = 4;
+    using Roles = TcRoles<T, MP>;
+    constexpr int kMmaWarp = Roles::kMmaWarp, kMmaWarpB = Roles::kMmaWarpB, kDrainWarp0 = Roles::kDrainWarp0;
+    constexpr int kTcThreads = Roles::kThreads;
     const bool is_drain = warp >= kDrainWarp0 && warp < kDrainWarp0 + 4;
     const bool is_mma = warp == kMmaWarp || warp == kMmaWarpB;
 
@@ -398,7 +422,7 @@ gram_tc_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ p
         // a warp prefetches the item this many of its own items ahead into L2 (measured: helps bf16 storage a
         // little, costs fp32 storage more than it brings)
         constexpr int kTcPrefetchAhead = kBf16 ? QN_TC_PREFETCH_BF16 : QN_TC_PREFETCH_F32;
-        const int pw = warp < kMmaWarp ? warp : warp == 8 ? 3 : warp - 6;  // warps 0-2, 8, 10-15 -> 0..9
+        const int pw = Roles::producer_index(warp);
         const int team = pw / kTeam, half = pw % kTeam;
         const int rq = lane / CPI, cl = lane % CPI;
         const int w0 = half * Shape::kRowsPerWarp + rq * RPL;  // first Worker of this lane's rows
@@ -670,7 +694,7 @@ static cudaError_t launch_tc(const T* g, int64_t n, int m, double* partials, int
     const size_t smem = sizeof(TcSmem<MP>) + 1024;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kern<<<grid, kTcThreads, smem, st>>>(g, n, m, partials, error_word);
+    kern<<<grid, TcRoles<T, MP>::kThreads, smem, st>>>(g, n, m, partials, error_word);
     return cudaGetLastError();
 }
 
