@@ -1,6 +1,6 @@
 """GPU parity: the CUDA library, called through its C ABI, against the fp64 CPU oracle on the same bits.
 
-Tolerances (stated by the task for this method): the cut-off j exact; theta_new within a relative L2
+Tolerances: the cut-off j exact; theta_new within a relative L2
 error of 1e-5 for fp32 storage and 2e-3 for bf16 storage (the bf16 figure is dominated by the single
 rounding of the output, about 1.5e-3); sigma within 1e-5 of sigma_1 for every k and within a relative
 1e-5 for the retained k <= j.
