@@ -590,13 +590,14 @@ def test_config2_full_size_sampled(qn):
     assert j == cfg.m - 1
 
 
-def test_config4_full_size_by_tiling(qn):
-    """Config 4 at its full n = 2^28, m = 64, bf16 (68.7 GB of inputs) is beyond what the oracle can read in a
-    test.  Property used instead: if the columns repeat with period p, the Gram is (n/p) times the block's Gram,
+@pytest.mark.parametrize("m", W.CONFIG4_M_SWEEP)
+def test_config4_full_size_by_tiling(qn, m):
+    """Config 4 at its full n = 2^28, bf16, at every m of its sweep as bench.py launches it (m = 64: 68.7 GB of
+    inputs) is beyond what the oracle can read in a test.  Property used instead: if the columns repeat with period p, the Gram is (n/p) times the block's Gram,
     so sigma scales by sqrt(n/p), j is unchanged and theta_new repeats with the block's values.  The block
     (p = 2^18 columns) goes through the oracle; the full-size input goes through the library."""
     free, _ = torch.cuda.mem_get_info()
-    cfg = W.CONFIGS[4]
+    cfg = W.CONFIGS[4].with_shape(m=m)
     need = 2 * cfg.m * cfg.n * 2 + cfg.n * 2 + (2 << 30)
     if free < need:
         pytest.skip("needs %.0f GB of free device memory" % (need / 1e9))
