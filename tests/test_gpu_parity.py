@@ -590,6 +590,38 @@ def test_config2_full_size_sampled(qn):
     assert j == cfg.m - 1
 
 
+def test_config3_full_size_sampled(qn):
+    """Config 3 at its full n = 124 M, m = 8, bf16, as bench.py launches it: the window is filled, then two
+    single-Worker Writes replace the oldest columns (bulk-copy row refresh), with an update after the fill and
+    after each Write.  j and sigma from the oracle's full passes over the window's bits, theta_new on sampled
+    columns."""
+    cfg = W.CONFIGS[3]
+    n, m = cfg.n, cfg.m
+    out = torch.empty(n, dtype=cfg.torch_dtype, device="cuda")
+    win_t = np.zeros((m, n), dtype=np.uint16)
+    win_g = np.zeros_like(win_t)
+    rng = np.random.default_rng(11)
+    idx = np.unique(np.concatenate([[0, 1, 7, 8, 2047, 2048, n - 1, n - 8, n - 9], rng.integers(0, n, 4096)])).astype(np.int64)
+    with qn.qn_create(n, m, cfg.torch_dtype) as h:
+        for t in range(m + 2):
+            th, gr = W.write_column(cfg, t, "cuda")
+            slot = t % m
+            qn.qn_push(h, -1, th, gr)
+            win_t[slot], win_g[slot] = W.to_bits(th), W.to_bits(gr)
+            del th, gr
+            if t < m - 1:
+                continue
+            j, sigma, status = qn.qn_update_window(h, cfg.tau, cfg.lam, out)
+            assert h.last_launches == 2
+            if t in (m - 1, m + 1):
+                ref = oracle.update(win_t, win_g, cfg.tau, cfg.lam, sample_idx=idx)
+                assert status == 0 and j == ref.j == m - 1
+                assert np.max(np.abs(np.array(sigma) - ref.sigma)) <= 1e-5 * ref.sigma[0]
+                assert np.max(np.abs(np.array(sigma)[:j] - ref.sigma[:j]) / ref.sigma[:j]) <= 1e-5
+                got = oracle.storage_to_f64(W.to_bits(out))[idx]
+                assert np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL["bf16"]
+
+
 @pytest.mark.parametrize("m", W.CONFIG4_M_SWEEP)
 def test_config4_full_size_by_tiling(qn, m):
     """Config 4 at its full n = 2^28, bf16, at every m of its sweep as bench.py launches it (m = 64: 68.7 GB of
