@@ -211,6 +211,16 @@ QN_API qn_status qn_update_host(qn_handle h, const void* theta_host, const void*
 /* Wait for the stream last used with this handle and return the deferred device status. */
 QN_API qn_status qn_status_sync(qn_handle h);
 
+/*
+ * Self-test of the device-side failure reporting (the paper has no counterpart).  Every wait inside the streaming
+ * kernels (on a bulk copy, a stage of the operand ring, a tensor-core commit) is bounded: when its poll limit runs
+ * out the kernel stops waiting, marks its partial sums invalid, sets a device word and returns, and the next
+ * eigen-solve reports QN_ERR_DEVICE_TIMEOUT.  This call enqueues a one-warp kernel that waits, with the same
+ * routine, on a barrier that nothing ever arrives on (the limit is one second), and sets that word: the next step on the
+ * handle then reports QN_ERR_DEVICE_TIMEOUT, and the one after it is clean again.  Nothing else is touched.
+ */
+QN_API qn_status qn_selftest_bounded_wait(qn_handle h, void* cuda_stream);
+
 /* Number of kernels this handle launched in its most recent qn_* call, and since creation. */
 QN_API int32_t qn_last_launches(qn_handle h);
 QN_API int64_t qn_total_launches(qn_handle h);

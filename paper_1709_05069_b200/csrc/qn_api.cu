@@ -616,6 +616,13 @@ extern "C" qn_status qn_status_sync(qn_handle h) {
     return fetch_result(h, h->last_stream, nullptr, nullptr);
 }
 
+extern "C" qn_status qn_selftest_bounded_wait(qn_handle h, void* cuda_stream) {
+    if (!h) return QN_ERR_INVALID;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return QN_ERR_CUDA;
+    return qn_launch_wait_probe(h->error_word, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? QN_OK : QN_ERR_CUDA;
+}
+
 extern "C" int32_t qn_last_launches(qn_handle h) { return h ? h->last_launches : 0; }
 extern "C" int64_t qn_total_launches(qn_handle h) { return h ? h->total_launches : 0; }
 extern "C" int32_t qn_last_sweeps(qn_handle h) { return h ? h->last_sweeps : -1; }

@@ -75,7 +75,14 @@ __device__ __forceinline__ double warp_sum(double x) {
 
 
 // ---- mbarrier helpers (shared memory barriers that track arrivals and bytes of bulk copies) -------------
-constexpr uint32_t kWaitLimit = 1u << 24;  // polls per wait before giving up (each poll may suspend ~1 us)
+constexpr uint32_t kWaitLimit = 1u << 24;         // polls per wait before giving up, whatever the clock says
+constexpr uint64_t kWaitLimitNs = 1000000000ull;  // and one second by the global timer, checked every 256 polls
+
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -100,12 +107,16 @@ template <bool kBackOff = true>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
     if (mbar_try(bar, parity)) return true;  // the common case costs one shared-memory round trip
     if (*abort) return false;
+    const uint64_t t0 = global_timer_ns();
     for (uint32_t it = 0; it < kWaitLimit; ++it) {
         if (mbar_try(bar, parity)) return true;
         // waiting warps sleep between polls so that they do not take issue slots from the others (a warp on the
         // critical path polls without sleeping)
         if (kBackOff) __nanosleep(64);
-        if ((it & 255u) == 255u && *abort) return false;
+        if ((it & 255u) == 255u) {
+            if (*abort) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) break;
+        }
     }
     *abort = 1;
     return false;

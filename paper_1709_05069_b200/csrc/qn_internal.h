@@ -79,6 +79,7 @@ struct qn_solve_params {
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
                            int* num_partials, int max_partials, cudaStream_t st, int* launches,
                            int* error_word = nullptr, double lambda_hint = 0.0);
+cudaError_t qn_launch_wait_probe(int* error_word, cudaStream_t st);
 bool qn_gram_tc_applicable(qn_dtype dtype, const void* g, int64_t n, int m);
 cudaError_t qn_launch_gram_tc(qn_dtype dtype, const void* g, int64_t n, int m, double* partials, int* num_partials,
                               int max_partials, int* error_word, cudaStream_t st);

@@ -366,6 +366,30 @@ static cudaError_t launch_row_t(const T* window_g, const T* g_col, T* window_row
 
 }  // namespace qn
 
+// Self-test of the bounded waits: one warp waits, with the library's own wait routine, on an mbarrier that nothing
+// ever arrives on.  The wait runs out after its limit (one second), the CTA reports through the error
+// word exactly as the streaming kernels do, and returns; the context stays usable.
+namespace qn {
+__global__ void __launch_bounds__(32) wait_probe_kernel(int* error_word) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    const bool ok = mbar_wait(&bar, 0u, &abort_flag);
+    __syncwarp();
+    if (threadIdx.x == 0 && !ok && error_word) atomicExch(error_word, 1);
+}
+}  // namespace qn
+
+cudaError_t qn_launch_wait_probe(int* error_word, cudaStream_t st) {
+    qn::wait_probe_kernel<<<1, 32, 0, st>>>(error_word);
+    return cudaGetLastError();
+}
+
 cudaError_t qn_launch_row(qn_dtype dtype, const void* window_g, const void* g_col, void* window_row_out,
                           const void* theta_col, void* theta_row_out, int64_t n, int m, int slot, double* partials,
                           int max_partials, double* raw_gram, double* dots_out, unsigned int* ticket, int* error_word,

@@ -25,7 +25,7 @@ EXPORTS = (
     "qn_strerror", "qn_create", "qn_destroy", "qn_update", "qn_gram", "qn_update_from_gram", "qn_apply_hinv", "qn_set_rank_cap", "qn_set_tau_cap", "qn_last_tau", "qn_push", "qn_update_window", "qn_rebuild",
     "qn_window_alloc", "qn_window_theta", "qn_window_g", "qn_window_mark_full", "qn_update_host", "qn_status_sync",
     "qn_last_launches", "qn_total_launches", "qn_last_sweeps", "qn_timing_begin", "qn_timing_end",
-    "qn_gram_static",
+    "qn_gram_static", "qn_selftest_bounded_wait",
 )
 TIME_KINDS = ("gram", "solve", "combine", "row")
 
@@ -50,6 +50,7 @@ def lib() -> ctypes.CDLL:
         L.qn_destroy.argtypes, L.qn_destroy.restype = [vp], i32
         L.qn_update.argtypes, L.qn_update.restype = [vp, vp, vp, dbl, dbl, vp, vp, vp, vp], i32
         L.qn_gram.argtypes, L.qn_gram.restype = [vp, vp, vp, vp], i32
+        L.qn_selftest_bounded_wait.argtypes, L.qn_selftest_bounded_wait.restype = [vp, vp], i32
         L.qn_set_tau_cap.argtypes, L.qn_set_tau_cap.restype = [vp, i32], i32
         L.qn_last_tau.argtypes, L.qn_last_tau.restype = [vp], dbl
         L.qn_set_rank_cap.argtypes, L.qn_set_rank_cap.restype = [vp, i32], i32
@@ -305,6 +306,11 @@ def qn_update_host(h: Handle, theta_host: torch.Tensor, g_host: torch.Tensor, ta
                               theta_new_host.data_ptr(), jp, sp, _stream_ptr(stream))
     _check(st, "qn_update_host", allow)
     return j.value, list(sigma), st
+
+
+def qn_selftest_bounded_wait(h: Handle, stream=None) -> None:
+    """Enqueue the bounded-wait self-test: the next step on ``h`` reports QN_ERR_DEVICE_TIMEOUT."""
+    _check(lib().qn_selftest_bounded_wait(h.ptr, _stream_ptr(stream)), "qn_selftest_bounded_wait")
 
 
 def qn_status_sync(h: Handle) -> int:

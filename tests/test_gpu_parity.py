@@ -491,6 +491,24 @@ def test_sharded_step_matches_the_whole_problem(qn, dtype, m, n, shards):
     assert np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL[dtype]
 
 
+def test_bounded_wait_runs_out_and_is_reported(qn):
+    """A device wait that nothing ends: the library's wait routine gives up after its poll limit, the kernel returns,
+    the next step reports QN_ERR_DEVICE_TIMEOUT, the context stays usable and the step after it is clean."""
+    cfg = W.CONFIGS[0]
+    theta, g = W.generate(cfg, "cuda")
+    out = torch.empty(cfg.n, dtype=cfg.torch_dtype, device="cuda")
+    ref = oracle.update(W.to_bits(theta), W.to_bits(g), cfg.tau, cfg.lam)
+    with qn.qn_create(cfg.n, cfg.m, cfg.torch_dtype) as h:
+        qn.qn_selftest_bounded_wait(h)
+        j, sigma, status = qn.qn_update(h, theta, g, cfg.tau, cfg.lam, out, allow=(qn.QN_ERR_DEVICE_TIMEOUT,))
+        assert status == qn.QN_ERR_DEVICE_TIMEOUT
+        assert bool(torch.isfinite(out).all())
+        j, sigma, status = qn.qn_update(h, theta, g, cfg.tau, cfg.lam, out)
+        assert status == 0 and j == ref.j
+        got = oracle.storage_to_f64(W.to_bits(out))
+        assert np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL["f32"]
+
+
 # --------------------------------------------------------------------------- bulk-copy Gram path (n >= 2^22, m <= 8)
 @pytest.mark.parametrize("dtype,m,n,gap", [
     ("bf16", 8, (1 << 22) + 8 * 3, True),    # config 4's first sweep point: short last tile
