@@ -28,7 +28,13 @@
  *
  * Streams.  `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  * Calls enqueue work on that stream and return without waiting unless they have to hand a HOST
- * result back (j_out / sigma_out non-NULL, qn_status_sync, qn_update_host).
+ * result back (j_out / sigma_out non-NULL, qn_status_sync, qn_update_host).  All calls on one handle
+ * share its workspace (partial sums, coefficients, result block): they must be ordered on the device,
+ * i.e. issued on one stream or on streams that the caller orders with events.  Two steps of one handle
+ * that overlap on the GPU race; use one handle per concurrent stream.
+ *
+ * Devices.  Every DEVICE pointer must point into memory of the handle's device (or managed memory);
+ * a host pointer or another GPU's memory is refused with QN_ERR_INVALID before anything is launched.
  *
  * Errors.  Every call returns a qn_status; nothing throws or aborts.  Arguments are validated on
  * the host before anything is launched.  Conditions only the device can see (a non-finite Gram,
@@ -98,6 +104,10 @@ QN_API qn_status qn_destroy(qn_handle h);
  * relative 1e-5; theta_new within a relative L2 error of 1e-5 (fp32 storage) or 2e-3 (bf16 storage: the single
  * rounding of the output).  The arithmetic of the Gram pass is chosen from n, m, the storage type and lambda
  * (fp64 products below 2^22 parameters; fp32 or tensor-core products above), never from the data.
+ * Condition on the sigma figures above 2^22 parameters: there the products are rounded (fp32, or for m > 8 and
+ * fp32 storage the 16 leading bits of each centred value on the tensor cores), and the bound relies on these
+ * rounding errors adding up like independent ones over the n columns (error of a retained sigma_k about
+ * 1e-5 sigma_1 / sqrt(n) per unit of 1 / lambda).  qn_set_gram_path(QN_GRAM_PATH_PLAIN_ALU) keeps fp32 products.
  */
 QN_API qn_status qn_update(qn_handle h, const void* theta, const void* g, double tau, double lambda,
                     void* theta_new, int32_t* j_out, double* sigma_out, void* cuda_stream);
@@ -110,6 +120,26 @@ QN_API qn_status qn_update(qn_handle h, const void* theta, const void* g, double
  * number can also be bounded directly.  sigma is still reported in full.  Host-side setting, no device work.
  */
 QN_API qn_status qn_set_rank_cap(qn_handle h, int32_t j_cap);
+
+/*
+ * Limit on the fp64 Jacobi sweeps of the eigen-solve (Section 2 leaves the eigen-solver open; this library uses
+ * cyclic Jacobi with a built-in limit of 30 sweeps, far above the 2 to 10 it needs).  max_sweeps = 0 restores the
+ * built-in limit.  A step that reaches the limit before every off-diagonal entry is below 1e-15 of the matrix
+ * norm still writes theta_new, j and sigma from the matrix as it stands and reports QN_ERR_NOT_CONVERGED.  Use:
+ * a bound on the step's latency, and a way to see that status in a test.  Host-side setting, no device work.
+ */
+QN_API qn_status qn_set_sweep_limit(qn_handle h, int32_t max_sweeps);
+
+/*
+ * Which kernels the Gram pass may use (the paper has no counterpart; for A/B measurements and tests).
+ *   QN_GRAM_PATH_AUTO       the default: tensor-core kernel for m > 8, bulk-copy kernel for m <= 8, both from
+ *                           2^22 parameters on aligned rows; the register-fed plain-ALU kernels elsewhere
+ *   QN_GRAM_PATH_PLAIN_ALU  the register-fed plain-ALU kernels everywhere (same results within the stated accuracy)
+ * Host-side setting of the handle; nothing is read from the environment.
+ */
+#define QN_GRAM_PATH_AUTO 0
+#define QN_GRAM_PATH_PLAIN_ALU 1
+QN_API qn_status qn_set_gram_path(qn_handle h, int32_t path);
 
 /*
  * Learning-rate cap (Section 3, last paragraph: the optimal rate is 1 / sigma_max of the Hessian, and the method
@@ -177,6 +207,10 @@ QN_API qn_status qn_update_from_gram(qn_handle h, const void* theta, const void*
  * slot's Gram row and column in O(m n); the paper is silent on which pair a Write replaces:
  * slot = -1 replaces the oldest, 0 <= slot < m replaces that slot.
  *   theta_col, g_col   [n] each, read-only
+ * slot = -1 moves on to the next-oldest pair only when the Write was enqueued (a call that fails on the host
+ * leaves the window and its order as they were).  If a later step reports QN_ERR_DEVICE_TIMEOUT, the row refresh
+ * of the most recent Write may be incomplete (its Gram row holds NaN, so every later update would report
+ * QN_ERR_NONFINITE and fall back to the SGD step): push that Write again into the same slot and call qn_rebuild.
  */
 QN_API qn_status qn_push(qn_handle h, int32_t slot, const void* theta_col, const void* g_col, void* cuda_stream);
 
@@ -246,8 +280,16 @@ QN_API int32_t qn_last_sweeps(qn_handle h);
  * The call makes no cudaMalloc/cudaFree and calls no allocating routine; it only enqueues two
  * kernels on cuda_stream and returns.
  *
- * First call on each device: looks up the array's device address (and raises one kernel's
- * shared-memory limit).  Make that first call during start-up, before any stream capture.
+ * First call on each device: looks up the array's device address and loads every kernel variant the
+ * entry point can dispatch to (whatever dtype, m, n and alignment later calls have) into the context,
+ * raising their shared-memory limits; loading code may allocate device memory inside the driver.
+ * Make that first call during start-up, before any stream capture; later calls of any shape load and
+ * allocate nothing.
+ *
+ * Failure reporting: there is no handle to carry a device status.  If one of the pass's bounded device
+ * waits runs out (see qn_selftest_bounded_wait), the call has already returned QN_OK and the only sign
+ * is that gram_out holds NaN; non-finite input shows the same way.  Check gram_out for finiteness
+ * where that matters.
  *
  * Sharing: all calls on a device use the same array, and it keeps whatever the previous call left
  * there.  Each call overwrites every entry it later reads, so nothing needs clearing and results

@@ -5,6 +5,8 @@
 
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "qn_internal.h"
 
 struct qn_ctx {
@@ -23,6 +25,8 @@ struct qn_ctx {
     int* error_word;              // device, set by a kernel that gave up on a bounded wait
     double* rhs;                  // device, m doubles: g_k^T z of qn_apply_hinv
     int32_t j_cap;                // < 0: none
+    int32_t sweep_limit;          // limit on the fp64 Jacobi sweeps, 0 = the built-in one
+    int32_t plain_alu;            // Gram pass restricted to the plain-ALU kernels (qn_set_gram_path)
     int32_t tau_cap;              // learning-rate cap on/off (qn_update and qn_update_host)
     double* partials_theta;       // device, as `partials`, allocated when the cap is first switched on
     double last_tau;              // learning rate of the most recent step whose results were fetched
@@ -38,6 +42,8 @@ struct qn_ctx {
     void* stage_theta;
     void* stage_g;
     void* stage_out;
+    cudaStream_t copy_stream;     // carries theta's host-to-device copy while the Gram pass runs
+    cudaEvent_t ev_fork, ev_theta;
 
     // optional per-kernel timing with CUDA events on the launching stream
     cudaEvent_t* ev;       // 2 events per timed kernel
@@ -93,12 +99,15 @@ struct DeviceGuard {
 
 inline bool finite_d(double x) { return isfinite(x); }
 
-// Brackets one kernel launch with two events when timing is on (see qn_timing_begin).
+// Brackets one kernel launch with an NVTX range (visible to a profiler, free without one) and, when timing is on
+// (see qn_timing_begin), with two events.
 struct KernelTimer {
     qn_handle h;
     cudaStream_t st;
     int idx = -1;
     KernelTimer(qn_handle h_, cudaStream_t st_, int kind) : h(h_), st(st_) {
+        static const char* const names[QN_TIME_KINDS] = {"qn:gram", "qn:solve", "qn:combine", "qn:row"};
+        nvtxRangePushA(names[kind]);
         if (h->ev && h->ev_used < h->ev_cap) {
             idx = h->ev_used++;
             h->ev_kind[idx] = kind;
@@ -107,6 +116,7 @@ struct KernelTimer {
     }
     ~KernelTimer() {
         if (idx >= 0) cudaEventRecord(h->ev[2 * idx + 1], st);
+        nvtxRangePop();
     }
 };
 
@@ -135,32 +145,50 @@ qn_status check_step_args(qn_handle h, double tau, double lambda, const void* th
     return QN_OK;
 }
 
+// A pointer the kernels of this handle may dereference: device memory of the handle's device, or managed memory.
+// Anything else (host memory, another GPU's memory) would fault on the device, so it is refused on the host.
+bool on_device(const void* p, int dev) {
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, p) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    if (a.type == cudaMemoryTypeManaged) return true;
+    return a.type == cudaMemoryTypeDevice && a.device == dev;
+}
+
 bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
     const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
     return a0 < b0 + nb && b0 < a0 + na;
 }
 
 // Gram partials -> solve -> combine on device buffers.
+// theta_ready (may be NULL): an event the stream waits for before the first kernel that reads theta.
 qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, double lambda, void* theta_new,
-                   cudaStream_t st) {
+                   cudaStream_t st, cudaEvent_t theta_ready = nullptr) {
     int np = 0;
     {
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st,
-                           &h->last_launches, h->error_word, lambda) != cudaSuccess)
+                           &h->last_launches, h->error_word, lambda, h->plain_alu != 0) != cudaSuccess)
             return QN_ERR_CUDA;
     }
     int np_theta = 0;
     if (h->tau_cap && h->partials_theta) {
         // the learning-rate cap needs ||Theta v_k||: one more Gram pass, over theta
+        if (theta_ready) {
+            if (cudaStreamWaitEvent(st, theta_ready, 0) != cudaSuccess) return QN_ERR_CUDA;
+            theta_ready = nullptr;
+        }
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, theta, h->n, h->m, false, h->partials_theta, &np_theta, h->max_partials, st,
-                           &h->last_launches, h->error_word, lambda) != cudaSuccess)
+                           &h->last_launches, h->error_word, lambda, h->plain_alu != 0) != cudaSuccess)
             return QN_ERR_CUDA;
     }
     qn_solve_params p;
     memset(&p, 0, sizeof(p));
     p.j_cap = h->j_cap;
+    p.max_sweeps = h->sweep_limit;
     p.tau_cap = h->tau_cap && h->partials_theta;
     p.partials_theta = h->partials_theta;
     p.num_partials_theta = np_theta;
@@ -177,6 +205,7 @@ qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, do
         KernelTimer t(h, st, QN_TIME_SOLVE);
         if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) return QN_ERR_CUDA;
     }
+    if (theta_ready && cudaStreamWaitEvent(st, theta_ready, 0) != cudaSuccess) return QN_ERR_CUDA;
     {
         KernelTimer t(h, st, QN_TIME_COMBINE);
         if (qn_launch_combine(h->dtype, theta, g, h->n, h->m, h->coef, theta_new, st, &h->last_launches) !=
@@ -269,6 +298,11 @@ extern "C" qn_status qn_destroy(qn_handle h) {
     cudaFree(h->stage_g);
     cudaFree(h->stage_out);
     if (h->host_result) cudaFreeHost(h->host_result);
+    if (h->copy_stream) {
+        cudaStreamDestroy(h->copy_stream);
+        cudaEventDestroy(h->ev_fork);
+        cudaEventDestroy(h->ev_theta);
+    }
     if (h->ev) {
         for (int i = 0; i < 2 * h->ev_cap; ++i) cudaEventDestroy(h->ev[i]);
         free(h->ev);
@@ -303,6 +337,18 @@ extern "C" qn_status qn_set_rank_cap(qn_handle h, int32_t j_cap) {
     return QN_OK;
 }
 
+extern "C" qn_status qn_set_sweep_limit(qn_handle h, int32_t max_sweeps) {
+    if (!h || max_sweeps < 0) return QN_ERR_INVALID;
+    h->sweep_limit = max_sweeps;
+    return QN_OK;
+}
+
+extern "C" qn_status qn_set_gram_path(qn_handle h, int32_t path) {
+    if (!h || (path != QN_GRAM_PATH_AUTO && path != QN_GRAM_PATH_PLAIN_ALU)) return QN_ERR_INVALID;
+    h->plain_alu = path == QN_GRAM_PATH_PLAIN_ALU;
+    return QN_OK;
+}
+
 extern "C" qn_status qn_update(qn_handle h, const void* theta, const void* g, double tau, double lambda,
                                void* theta_new, int32_t* j_out, double* sigma_out, void* cuda_stream) {
     qn_status s = check_step_args(h, tau, lambda, theta_new);
@@ -313,6 +359,8 @@ extern "C" qn_status qn_update(qn_handle h, const void* theta, const void* g, do
         return QN_ERR_INVALID;
     DeviceGuard guard(h->device);
     if (!guard.ok) return QN_ERR_CUDA;
+    if (!on_device(theta, h->device) || !on_device(g, h->device) || !on_device(theta_new, h->device))
+        return QN_ERR_INVALID;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     begin_call(h, st);
     s = run_step(h, theta, g, tau, lambda, theta_new, st);
@@ -333,11 +381,15 @@ extern "C" qn_status qn_update_from_gram(qn_handle h, const void* theta, const v
         return QN_ERR_INVALID;
     DeviceGuard guard(h->device);
     if (!guard.ok) return QN_ERR_CUDA;
+    if (!on_device(theta, h->device) || !on_device(g, h->device) || !on_device(theta_new, h->device) ||
+        !on_device(gram, h->device))
+        return QN_ERR_INVALID;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     begin_call(h, st);
     qn_solve_params p;
     memset(&p, 0, sizeof(p));
     p.j_cap = h->j_cap;
+    p.max_sweeps = h->sweep_limit;
     p.m = h->m;
     p.source = QN_SRC_SUMMED;
     p.raw_gram = const_cast<double*>(gram);  // read only in this mode
@@ -373,6 +425,9 @@ extern "C" qn_status qn_apply_hinv(qn_handle h, const void* theta, const void* g
         return QN_ERR_INVALID;
     DeviceGuard guard(h->device);
     if (!guard.ok) return QN_ERR_CUDA;
+    if (!on_device(theta, h->device) || !on_device(g, h->device) || !on_device(z, h->device) ||
+        !on_device(out, h->device))
+        return QN_ERR_INVALID;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     begin_call(h, st);
     // 1. g_k^T z for every Worker (the row pass of the asynchronous mode with z in the place of the new column;
@@ -389,13 +444,14 @@ extern "C" qn_status qn_apply_hinv(qn_handle h, const void* theta, const void* g
     if (s == QN_OK) {
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st, &h->last_launches,
-                           h->error_word, lambda) != cudaSuccess)
+                           h->error_word, lambda, h->plain_alu != 0) != cudaSuccess)
             s = QN_ERR_CUDA;
     }
     if (s == QN_OK) {
         qn_solve_params p;
         memset(&p, 0, sizeof(p));
         p.j_cap = h->j_cap;
+        p.max_sweeps = h->sweep_limit;
         p.m = h->m;
         p.source = QN_SRC_PARTIALS;
         p.partials = h->partials;
@@ -424,17 +480,22 @@ extern "C" qn_status qn_gram(qn_handle h, const void* g, double* gram_out, void*
     if (!h || !g || !gram_out) return QN_ERR_INVALID;
     DeviceGuard guard(h->device);
     if (!guard.ok) return QN_ERR_CUDA;
+    if (!on_device(g, h->device) || !on_device(gram_out, h->device)) return QN_ERR_INVALID;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     begin_call(h, st);
     int np = 0;
     qn_status s = QN_OK;
-    if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st, &h->last_launches,
-                       h->error_word) != cudaSuccess)
-        s = QN_ERR_CUDA;
+    {
+        KernelTimer t(h, st, QN_TIME_GRAM);
+        if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st, &h->last_launches,
+                           h->error_word, 0.0, h->plain_alu != 0) != cudaSuccess)
+            s = QN_ERR_CUDA;
+    }
     if (s == QN_OK) {
         qn_solve_params p;
         memset(&p, 0, sizeof(p));
         p.j_cap = h->j_cap;
+        p.max_sweeps = h->sweep_limit;
         p.m = h->m;
         p.source = QN_SRC_PARTIALS;
         p.partials = h->partials;
@@ -445,6 +506,7 @@ extern "C" qn_status qn_gram(qn_handle h, const void* g, double* gram_out, void*
         p.lambda = 1.0;
         p.coef = h->coef;
         p.result = h->result;
+        KernelTimer t(h, st, QN_TIME_SOLVE);
         if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) s = QN_ERR_CUDA;
     }
     end_call(h);
@@ -477,12 +539,11 @@ extern "C" qn_status qn_push(qn_handle h, int32_t slot, const void* theta_col, c
     const size_t col_bytes = (size_t)h->n * h->elem, win_bytes = col_bytes * h->m;
     if (overlaps(theta_col, col_bytes, h->win_theta, win_bytes) || overlaps(g_col, col_bytes, h->win_g, win_bytes))
         return QN_ERR_INVALID;
+    if (!on_device(theta_col, h->device) || !on_device(g_col, h->device)) return QN_ERR_INVALID;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     begin_call(h, st);
-    if (slot < 0) {
-        slot = h->head;
-        h->head = (h->head + 1) % h->m;
-    }
+    const bool oldest = slot < 0;
+    if (oldest) slot = h->head;
     char* trow = static_cast<char*>(h->win_theta) + (size_t)slot * col_bytes;
     char* grow = static_cast<char*>(h->win_g) + (size_t)slot * col_bytes;
     bool theta_landed = false;
@@ -497,7 +558,10 @@ extern "C" qn_status qn_push(qn_handle h, int32_t slot, const void* theta_col, c
     if (s == QN_OK && !theta_landed &&
         cudaMemcpyAsync(trow, theta_col, col_bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
         s = QN_ERR_CUDA;
-    if (s == QN_OK) h->filled |= (1ull << slot);
+    if (s == QN_OK) {
+        h->filled |= (1ull << slot);
+        if (oldest) h->head = (h->head + 1) % h->m;  // a Write that could not be enqueued does not use up its slot
+    }
     end_call(h);
     return s;
 }
@@ -513,11 +577,13 @@ extern "C" qn_status qn_update_window(qn_handle h, double tau, double lambda, vo
         return QN_ERR_INVALID;
     DeviceGuard guard(h->device);
     if (!guard.ok) return QN_ERR_CUDA;
+    if (!on_device(theta_new, h->device)) return QN_ERR_INVALID;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     begin_call(h, st);
     qn_solve_params p;
     memset(&p, 0, sizeof(p));
     p.j_cap = h->j_cap;
+    p.max_sweeps = h->sweep_limit;
     p.m = h->m;
     p.source = QN_SRC_WINDOW;
     p.raw_gram = h->raw_gram;
@@ -558,6 +624,7 @@ extern "C" qn_status qn_rebuild(qn_handle h, void* cuda_stream) {
         qn_solve_params p;
         memset(&p, 0, sizeof(p));
         p.j_cap = h->j_cap;
+        p.max_sweeps = h->sweep_limit;
         p.m = h->m;
         p.source = QN_SRC_PARTIALS;
         p.partials = h->partials;
@@ -594,13 +661,29 @@ extern "C" qn_status qn_update_host(qn_handle h, const void* theta_host, const v
             return QN_ERR_ALLOC;
         }
     }
+    if (!h->copy_stream) {
+        bool ok = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&h->ev_theta, cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) {
+            cudaGetLastError();
+            return QN_ERR_CUDA;
+        }
+    }
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     begin_call(h, st);
-    // g first: the Gram pass needs only g, so theta's copy can overlap it on a copy engine
+    // g goes first on the caller's stream, since the Gram pass and the eigen-solve need only g.  theta's copy is
+    // enqueued on a second stream (ordered after the work already on the caller's stream: the staging may still be
+    // read by an earlier step), so it runs behind g's copy on the link and overlaps the Gram pass and the solve; the
+    // caller's stream waits for it just before the pass that reads theta.
     if (cudaMemcpyAsync(h->stage_g, g_host, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) s = QN_ERR_CUDA;
-    if (s == QN_OK && cudaMemcpyAsync(h->stage_theta, theta_host, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    if (s == QN_OK && (cudaEventRecord(h->ev_fork, st) != cudaSuccess ||
+                       cudaStreamWaitEvent(h->copy_stream, h->ev_fork, 0) != cudaSuccess ||
+                       cudaMemcpyAsync(h->stage_theta, theta_host, in_bytes, cudaMemcpyHostToDevice, h->copy_stream) !=
+                           cudaSuccess ||
+                       cudaEventRecord(h->ev_theta, h->copy_stream) != cudaSuccess))
         s = QN_ERR_CUDA;
-    if (s == QN_OK) s = run_step(h, h->stage_theta, h->stage_g, tau, lambda, h->stage_out, st);
+    if (s == QN_OK) s = run_step(h, h->stage_theta, h->stage_g, tau, lambda, h->stage_out, st, h->ev_theta);
     if (s == QN_OK &&
         cudaMemcpyAsync(theta_new_host, h->stage_out, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         s = QN_ERR_CUDA;

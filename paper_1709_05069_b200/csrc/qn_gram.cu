@@ -17,8 +17,6 @@
 //             carry the cancellation of the later m x m centring.
 // Every thread owns fixed columns and fixed output entries, so results are bitwise reproducible for
 // a given grid.
-#include <stdlib.h>
-
 #include "qn_device.cuh"
 
 namespace qn {
@@ -733,22 +731,16 @@ static cudaError_t launch_gram_t(const T* g, int64_t n, int m, bool raw, double*
 
 }  // namespace qn
 
-// QN_GRAM_PATH=alu forces the plain-ALU kernels (for A/B measurements); anything else lets the
-// tensor-core kernel take the cases it covers.
-static bool tc_allowed() {
-    const char* v = getenv("QN_GRAM_PATH");
-    return !(v && v[0] == 'a');
-}
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
                            int* num_partials, int max_partials, cudaStream_t st, int* launches, int* error_word,
-                           double lambda_hint) {
+                           double lambda_hint, bool plain_alu) {
     cudaError_t e;
     const int64_t elem = dtype == QN_F32 ? 4 : 2;
-    if (!raw && tc_allowed() && qn_gram_tc_applicable(dtype, g, n, m)) {
+    if (!raw && !plain_alu && qn_gram_tc_applicable(dtype, g, n, m)) {
         e = qn_launch_gram_tc(dtype, g, n, m, partials, num_partials, max_partials, error_word, st);
-    } else if (!raw && tc_allowed() && m <= qn::kDirectM && n >= QN_PRECISE_BELOW &&
+    } else if (!raw && !plain_alu && m <= qn::kDirectM && n >= QN_PRECISE_BELOW &&
                reinterpret_cast<uintptr_t>(g) % 16 == 0 && (n * elem) % 16 == 0) {
-        // bulk-copy variant of the direct kernel (QN_GRAM_PATH=alu keeps the register-fed one, for A/B runs)
+        // bulk-copy variant of the direct kernel (plain_alu keeps the register-fed one, for A/B runs)
         const bool ref0 = lambda_hint >= QN_REF0_MIN_LAMBDA;
         e = dtype == QN_F32 ? qn::launch_gram_stream(static_cast<const float*>(g), n, m, partials, num_partials,
                                                      max_partials, error_word, false, st)
@@ -761,5 +753,50 @@ cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool
                                     max_partials, st);
     }
     if (e == cudaSuccess && launches) *launches += 1;
+    return e;
+}
+
+namespace qn {
+template <typename K>
+static cudaError_t preload_kernel(K kern, size_t smem = 0) {
+    cudaFuncAttributes a;
+    cudaError_t e = cudaFuncGetAttributes(&a, kern);  // loads the kernel's code into the current context
+    if (e == cudaSuccess && smem) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    return e;
+}
+template <typename T, bool kAligned>
+static cudaError_t preload_alu() {
+    cudaError_t e = cudaSuccess;
+    if (e == cudaSuccess) e = preload_kernel(gram_direct_kernel<T, kAligned, kFast>);
+    if (e == cudaSuccess) e = preload_kernel(gram_direct_kernel<T, kAligned, kPrecise>);
+    if (e == cudaSuccess) e = preload_kernel(gram_direct_kernel<T, kAligned, kRaw>);
+    if (e == cudaSuccess) e = preload_kernel(gram_tiled_kernel<T, kAligned, kFast>, sizeof(TiledSmem));
+    if (e == cudaSuccess) e = preload_kernel(gram_tiled_kernel<T, kAligned, kPrecise>, sizeof(TiledSmem));
+    if (e == cudaSuccess) e = preload_kernel(gram_tiled_kernel<T, kAligned, kRaw>, sizeof(TiledSmem));
+    return e;
+}
+template <typename T>
+static cudaError_t preload_stream() {
+    const size_t smem = sizeof(GsSmem) + 128;
+    cudaError_t e = preload_kernel(gram_stream_kernel<T, 2, false>, smem);
+    if (e == cudaSuccess) e = preload_kernel(gram_stream_kernel<T, 4, false>, smem);
+    if (e == cudaSuccess) e = preload_kernel(gram_stream_kernel<T, 8, false>, smem);
+    if (e == cudaSuccess && sizeof(T) == 2) {
+        e = preload_kernel(gram_stream_kernel<T, 2, true>, smem);
+        if (e == cudaSuccess) e = preload_kernel(gram_stream_kernel<T, 4, true>, smem);
+        if (e == cudaSuccess) e = preload_kernel(gram_stream_kernel<T, 8, true>, smem);
+    }
+    return e;
+}
+}  // namespace qn
+
+cudaError_t qn_gram_preload() {
+    cudaError_t e = qn::preload_alu<float, true>();
+    if (e == cudaSuccess) e = qn::preload_alu<float, false>();
+    if (e == cudaSuccess) e = qn::preload_alu<__nv_bfloat16, true>();
+    if (e == cudaSuccess) e = qn::preload_alu<__nv_bfloat16, false>();
+    if (e == cudaSuccess) e = qn::preload_stream<float>();
+    if (e == cudaSuccess) e = qn::preload_stream<__nv_bfloat16>();
+    if (e == cudaSuccess) e = qn_gram_tc_preload();
     return e;
 }

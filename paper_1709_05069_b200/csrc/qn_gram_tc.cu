@@ -715,7 +715,28 @@ static cudaError_t launch_tc_any(const T* g, int64_t n, int m, double* partials,
     return launch_tc<T, 64>(g, n, m, partials, grid, error_word, st);
 }
 
+template <typename T, int MP>
+static cudaError_t preload_tc() {
+    const size_t smem = sizeof(TcSmem<MP>) + 1024;
+    cudaFuncAttributes a;
+    cudaError_t e = cudaFuncGetAttributes(&a, gram_tc_kernel<T, MP, true>);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gram_tc_kernel<T, MP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&a, gram_tc_kernel<T, MP, false>);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gram_tc_kernel<T, MP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    return e;
+}
+
 }  // namespace qn
+
+cudaError_t qn_gram_tc_preload() {
+    cudaError_t e = qn::preload_tc<float, 16>();
+    if (e == cudaSuccess) e = qn::preload_tc<float, 32>();
+    if (e == cudaSuccess) e = qn::preload_tc<float, 64>();
+    if (e == cudaSuccess) e = qn::preload_tc<__nv_bfloat16, 16>();
+    if (e == cudaSuccess) e = qn::preload_tc<__nv_bfloat16, 32>();
+    if (e == cudaSuccess) e = qn::preload_tc<__nv_bfloat16, 64>();
+    return e;
+}
 
 bool qn_gram_tc_applicable(qn_dtype dtype, const void* g, int64_t n, int m) {
     const int64_t elem = dtype == QN_F32 ? 4 : 2;

@@ -60,6 +60,7 @@ struct qn_solve_params {
     int32_t gram_only;    // stop after writing gram_out
     double tau, lambda;
     int32_t j_cap;        // < 0: no cap; else at most this many of the modes kept by the lambda rule
+    int32_t max_sweeps;   // limit on the fp64 Jacobi sweeps (0: the built-in limit); reaching it gives QN_ERR_NOT_CONVERGED
     int32_t tau_cap;      // != 0 with partials_theta: tau <- min(tau, 1 / max_k sigma_k / ||Theta v_k||)
     const double* partials_theta;  // Gram partials of theta (same layout as `partials`), or NULL
     int32_t num_partials_theta;
@@ -76,9 +77,14 @@ struct qn_solve_params {
 // bulk-copy kernel for bf16 storage and m <= 8 may take Worker 0 instead of the mean as its per-column reference
 // (a third fewer instructions; the error of a retained sigma_k grows as 1 / lambda^2, see qn_gram.cu).
 #define QN_REF0_MIN_LAMBDA 0.01
+// plain_alu: keep to the register-fed plain-ALU kernels (qn_set_gram_path; A/B measurements and tests).
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
                            int* num_partials, int max_partials, cudaStream_t st, int* launches,
-                           int* error_word = nullptr, double lambda_hint = 0.0);
+                           int* error_word = nullptr, double lambda_hint = 0.0, bool plain_alu = false);
+// Loads every Gram kernel variant into the current context (allocates nothing the caller can see later: after it,
+// the first launch of a variant no longer loads code).
+cudaError_t qn_gram_preload();
+cudaError_t qn_gram_tc_preload();
 cudaError_t qn_launch_wait_probe(int* error_word, cudaStream_t st);
 bool qn_gram_tc_applicable(qn_dtype dtype, const void* g, int64_t n, int m);
 cudaError_t qn_launch_gram_tc(qn_dtype dtype, const void* g, int64_t n, int m, double* partials, int* num_partials,

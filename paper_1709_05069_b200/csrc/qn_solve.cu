@@ -426,7 +426,8 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
             s = s0 * k;
         }
     };
-    while (!converged && sweeps < kMaxSweeps) {
+    const int sweep_limit = prm.max_sweeps > 0 && prm.max_sweeps < kMaxSweeps ? prm.max_sweeps : kMaxSweeps;
+    while (!converged && sweeps < sweep_limit) {
         for (int r = 0; r < N; ++r) {
             double x00 = 0.0, x01 = 0.0, x10 = 0.0, x11 = 0.0;
             if (worker) {

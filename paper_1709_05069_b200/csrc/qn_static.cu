@@ -35,7 +35,9 @@ qn_status scratch_for_current_device(double** out) {
             cudaGetLastError();
             return QN_ERR_CUDA;
         }
-        if (qn_solve_init() != cudaSuccess) {  // raises the solve kernel's shared-memory limit; allocates nothing
+        // Load every kernel this entry point can dispatch to, and raise their shared-memory limits, now: the first
+        // use of a kernel loads its code, which may allocate inside the driver, and later calls must not.
+        if (qn_solve_init() != cudaSuccess || qn_gram_preload() != cudaSuccess) {
             cudaGetLastError();
             return QN_ERR_CUDA;
         }

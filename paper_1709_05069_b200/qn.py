@@ -14,6 +14,8 @@ import torch
 QN_F32 = 0
 QN_BF16 = 1
 QN_MAX_M = 64
+QN_GRAM_PATH_AUTO = 0
+QN_GRAM_PATH_PLAIN_ALU = 1
 
 (QN_OK, QN_ERR_INVALID, QN_ERR_ALLOC, QN_ERR_CUDA, QN_ERR_STATE, QN_ERR_NOT_CONVERGED, QN_ERR_NONFINITE,
  QN_ERR_DEVICE_TIMEOUT) = range(8)
@@ -22,7 +24,9 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libqn.so")
 _lib: Optional[ctypes.CDLL] = None
 
 EXPORTS = (
-    "qn_strerror", "qn_create", "qn_destroy", "qn_update", "qn_gram", "qn_update_from_gram", "qn_apply_hinv", "qn_set_rank_cap", "qn_set_tau_cap", "qn_last_tau", "qn_push", "qn_update_window", "qn_rebuild",
+    "qn_strerror", "qn_create", "qn_destroy", "qn_update", "qn_gram", "qn_update_from_gram", "qn_apply_hinv",
+    "qn_set_rank_cap", "qn_set_sweep_limit", "qn_set_gram_path", "qn_set_tau_cap", "qn_last_tau", "qn_push",
+    "qn_update_window", "qn_rebuild",
     "qn_window_alloc", "qn_window_theta", "qn_window_g", "qn_window_mark_full", "qn_update_host", "qn_status_sync",
     "qn_last_launches", "qn_total_launches", "qn_last_sweeps", "qn_timing_begin", "qn_timing_end",
     "qn_gram_static", "qn_selftest_bounded_wait",
@@ -54,6 +58,8 @@ def lib() -> ctypes.CDLL:
         L.qn_set_tau_cap.argtypes, L.qn_set_tau_cap.restype = [vp, i32], i32
         L.qn_last_tau.argtypes, L.qn_last_tau.restype = [vp], dbl
         L.qn_set_rank_cap.argtypes, L.qn_set_rank_cap.restype = [vp, i32], i32
+        L.qn_set_sweep_limit.argtypes, L.qn_set_sweep_limit.restype = [vp, i32], i32
+        L.qn_set_gram_path.argtypes, L.qn_set_gram_path.restype = [vp, i32], i32
         L.qn_apply_hinv.argtypes, L.qn_apply_hinv.restype = [vp, vp, vp, dbl, vp, vp, vp, vp, vp], i32
         L.qn_update_from_gram.argtypes, L.qn_update_from_gram.restype = [vp, vp, vp, vp, dbl, dbl, vp, vp, vp, vp], i32
         L.qn_push.argtypes, L.qn_push.restype = [vp, i32, vp, vp, vp], i32
@@ -94,10 +100,11 @@ def dtype_code(dtype: torch.dtype) -> int:
 
 
 class Handle:
-    """Owner of a ``qn_handle``.  ``n``, ``m``, ``dtype`` as passed to ``qn_create``."""
+    """Owner of a ``qn_handle``.  ``n``, ``m``, ``dtype`` as passed to ``qn_create``; ``device`` is the index of
+    the CUDA device the handle lives on (every tensor passed with it must live there too)."""
 
-    def __init__(self, ptr: int, n: int, m: int, dtype: torch.dtype):
-        self.ptr, self.n, self.m, self.dtype = ptr, n, m, dtype
+    def __init__(self, ptr: int, n: int, m: int, dtype: torch.dtype, device: int = 0):
+        self.ptr, self.n, self.m, self.dtype, self.device = ptr, n, m, dtype, device
 
     def close(self):
         if self.ptr:
@@ -135,25 +142,35 @@ def _stream_ptr(stream) -> int:
     return int(stream.cuda_stream)
 
 
+def _same_device(t, h: Handle, name: str) -> None:
+    # a tensor on another GPU would make the kernels dereference memory they cannot reach
+    if t.device.index != h.device:
+        raise ValueError("%s lives on cuda:%s but the handle was created on cuda:%d" % (name, t.device.index, h.device))
+
+
 def _dev_matrix(t: torch.Tensor, h: Handle, name: str) -> int:
     if not t.is_cuda or t.dtype != h.dtype or tuple(t.shape) != (h.m, h.n) or not t.is_contiguous():
         raise ValueError("%s must be a contiguous CUDA tensor [m][n] of the handle's dtype" % name)
+    _same_device(t, h, name)
     return t.data_ptr()
 
 
 def _dev_vector(t: torch.Tensor, h: Handle, name: str) -> int:
     if not t.is_cuda or t.dtype != h.dtype or tuple(t.shape) != (h.n,) or not t.is_contiguous():
         raise ValueError("%s must be a contiguous CUDA tensor [n] of the handle's dtype" % name)
+    _same_device(t, h, name)
     return t.data_ptr()
 
 
 def qn_create(n: int, m: int, dtype: torch.dtype) -> Handle:
     """Handle on the current CUDA device (``torch.cuda.current_device()``)."""
     out = ctypes.c_void_p(0)
+    device = 0
     if torch.cuda.is_available():
-        torch.cuda.set_device(torch.cuda.current_device())  # make torch's device the runtime's current one
+        device = torch.cuda.current_device()
+        torch.cuda.set_device(device)  # make torch's device the runtime's current one
     _check(lib().qn_create(int(n), int(m), dtype_code(dtype), ctypes.byref(out)), "qn_create")
-    return Handle(out.value, int(n), int(m), dtype)
+    return Handle(out.value, int(n), int(m), dtype, device)
 
 
 def qn_destroy(h: Handle) -> None:
@@ -192,6 +209,17 @@ def qn_set_rank_cap(h: Handle, j_cap: Optional[int]) -> None:
     _check(lib().qn_set_rank_cap(h.ptr, -1 if j_cap is None else int(j_cap)), "qn_set_rank_cap")
 
 
+def qn_set_sweep_limit(h: Handle, max_sweeps: Optional[int]) -> None:
+    """Limit the fp64 Jacobi sweeps of later steps on this handle (``None`` or 0: the built-in limit of 30).  A step
+    that reaches the limit still writes its outputs and reports QN_ERR_NOT_CONVERGED."""
+    _check(lib().qn_set_sweep_limit(h.ptr, 0 if max_sweeps is None else int(max_sweeps)), "qn_set_sweep_limit")
+
+
+def qn_set_gram_path(h: Handle, path: int) -> None:
+    """``QN_GRAM_PATH_AUTO`` (default) or ``QN_GRAM_PATH_PLAIN_ALU`` (register-fed plain-ALU Gram kernels only)."""
+    _check(lib().qn_set_gram_path(h.ptr, int(path)), "qn_set_gram_path")
+
+
 def qn_set_tau_cap(h: Handle, on: bool) -> None:
     """Bound tau by the reciprocal of the method's estimate of the Hessian's largest singular value in later
     ``qn_update`` / ``qn_update_host`` calls on this handle (one more pass, over theta)."""
@@ -218,6 +246,7 @@ def qn_apply_hinv(h: Handle, theta: torch.Tensor, g: torch.Tensor, lam: float, z
 def _check_gram_buffer(h: Handle, gram: torch.Tensor) -> None:
     if not gram.is_cuda or gram.dtype != torch.float64 or gram.numel() != h.m * h.m + h.m or not gram.is_contiguous():
         raise ValueError("the Gram buffer must be a contiguous CUDA float64 tensor with m*m + m elements")
+    _same_device(gram, h, "the Gram buffer")
 
 
 def qn_update_from_gram(h: Handle, theta: torch.Tensor, g: torch.Tensor, gram: torch.Tensor, tau: float, lam: float,
@@ -253,13 +282,20 @@ def qn_update_sharded(h: Handle, theta: torch.Tensor, g: torch.Tensor, tau: floa
 
     ``theta``, ``g``: [m][n_local] of this rank; ``gram_buf``: CUDA float64 scratch with m*m + m elements.  The only
     exchange is one all-reduce of ``gram_buf`` (``torch.distributed``, NCCL between GPUs); every other byte stays on
-    its GPU.  With no initialised process group (or a world of one) this is ``qn_gram`` + ``qn_update_from_gram``."""
+    its GPU.  With no initialised process group this is ``qn_gram`` + ``qn_update_from_gram``; with a group of one
+    rank the all-reduce still runs (it is the identity).
+
+    The collective is ordered against torch's CURRENT stream, so the three calls run with ``stream`` made current:
+    the all-reduce then sits between the Gram pass and the step on the same stream."""
     import torch.distributed as dist
 
-    qn_gram(h, g, gram_buf, stream=stream)
-    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
-        dist.all_reduce(gram_buf, op=dist.ReduceOp.SUM, group=group)
-    return qn_update_from_gram(h, theta, g, gram_buf, tau, lam, theta_new, want_host=want_host, stream=stream)
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    with torch.cuda.stream(stream):
+        qn_gram(h, g, gram_buf, stream=stream)
+        if dist.is_available() and dist.is_initialized():
+            dist.all_reduce(gram_buf, op=dist.ReduceOp.SUM, group=group)
+        return qn_update_from_gram(h, theta, g, gram_buf, tau, lam, theta_new, want_host=want_host, stream=stream)
 
 
 def qn_push(h: Handle, slot: int, theta_col: torch.Tensor, g_col: torch.Tensor, stream=None) -> None:
@@ -344,5 +380,9 @@ def qn_gram_static(g: torch.Tensor, gram_out: torch.Tensor, stream=None) -> None
     if not gram_out.is_cuda or gram_out.dtype != torch.float64 or gram_out.numel() != m * m + m \
             or not gram_out.is_contiguous():
         raise ValueError("gram_out must be a contiguous CUDA float64 tensor with m*m + m elements")
-    _check(lib().qn_gram_static(int(n), int(m), dtype_code(g.dtype), g.data_ptr(), gram_out.data_ptr(),
-                                _stream_ptr(stream)), "qn_gram_static")
+    if gram_out.device != g.device:
+        raise ValueError("g and gram_out must live on the same device")
+    # the call runs on the runtime's current device: make that the tensors' device for its duration
+    with torch.cuda.device(g.device):
+        _check(lib().qn_gram_static(int(n), int(m), dtype_code(g.dtype), g.data_ptr(), gram_out.data_ptr(),
+                                    _stream_ptr(stream)), "qn_gram_static")

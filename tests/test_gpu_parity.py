@@ -11,10 +11,9 @@ import torch
 
 import oracle
 import workloads as W
+from gpu_helpers import TOL, Guarded, assert_gap, check_against_oracle, copy_device_bytes, run_gpu, window_bits
 
 pytestmark = pytest.mark.gpu
-
-TOL = {"f32": 1e-5, "bf16": 2e-3}
 
 
 @pytest.fixture(scope="module")
@@ -24,62 +23,6 @@ def qn():
     assert torch.cuda.is_available()
     mod.lib()
     return mod
-
-
-def run_gpu(qn, theta, g, tau, lam):
-    m, n = theta.shape
-    out = torch.empty(n, dtype=theta.dtype, device="cuda")
-    with qn.qn_create(n, m, theta.dtype) as h:
-        j, sigma, status = qn.qn_update(h, theta, g, tau, lam, out)
-        launches = h.last_launches
-    return out, j, np.array(sigma), status, launches
-
-
-def check_against_oracle(qn, theta, g, tau, lam, dtype, expect_j=None, sample=None):
-    out, j, sigma, status, launches = run_gpu(qn, theta, g, tau, lam)
-    tb, gb = W.to_bits(theta), W.to_bits(g)
-    ref = oracle.update(tb, gb, tau, lam, sample_idx=sample)
-    assert status == 0
-    assert launches == 3
-    assert j == ref.j, (j, ref.j, sigma / sigma[0], ref.sigma / ref.sigma[0])
-    if expect_j is not None:
-        assert j == expect_j
-    s1 = ref.sigma[0]
-    assert np.max(np.abs(sigma - ref.sigma)) <= 1e-5 * s1
-    if j:
-        assert np.max(np.abs(sigma[:j] - ref.sigma[:j]) / ref.sigma[:j]) <= 1e-5
-    got = oracle.storage_to_f64(W.to_bits(out))
-    if sample is not None:
-        got = got[sample]
-    rel = np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new)
-    if len(got) < 64:
-        # With a handful of elements the L2 figure is not an average.  Bound every element instead: the
-        # fp32 combination is accurate to 1e-5 of the magnitude of the terms it adds (thetabar, tau*z_perp
-        # and tau*sum alpha_k y_k / sigma_k, which may cancel), and for bf16 storage the single output
-        # rounding adds at most one bf16 ulp (2^-8 relative, 2^-133 absolute).
-        t64, g64 = oracle.storage_to_f64(tb), oracle.storage_to_f64(gb)
-        U, Y, sg, jj = oracle.left_vectors(tb, gb, lam)
-        al = ref.alpha[:jj]
-        scale = np.abs(t64.mean(0)) + abs(tau) * (np.abs(g64.mean(0)) + np.abs(U) @ np.abs(al)
-                                                  + np.abs(Y) @ np.abs(al / sg[:jj]))
-        if sample is not None:
-            scale = scale[sample]
-        bound = 1e-5 * scale
-        if dtype == "bf16":
-            bound = bound + 2.0 ** -8 * np.abs(ref.theta_new) + 2.0 ** -133
-        assert np.all(np.abs(got - ref.theta_new) <= bound), (got, ref.theta_new, bound)
-    else:
-        assert rel <= TOL[dtype], rel
-    return rel, j, out
-
-
-def assert_gap(theta, g, lam):
-    """The generator's promise: a clear gap around lam*sigma_1 in fp64 on the rounded data."""
-    ref = oracle.update(W.to_bits(theta), W.to_bits(g), 1.0, lam, want_theta=False)
-    j, s = ref.j, ref.sigma
-    assert s[j - 1] >= 2 * lam * s[0]
-    assert s[j] <= lam * s[0] / 2
-    return j
 
 
 # --------------------------------------------------------------------------- the five configs' shapes
@@ -228,11 +171,13 @@ def test_gram_entry_point(qn, dtype, m, n):
     """qn_gram: centred Gram and w = G^T gbar against the oracle's Gram and a numpy product."""
     cfg = W.Config(13, n, m, dtype, -1, 1, 0, 0.05, 1e-3, 0.5, 0.05)
     theta, g = W.generate(cfg, "cuda")
-    buf = torch.empty(m * m + m, dtype=torch.float64, device="cuda")
+    guarded = Guarded(m * m + m, torch.float64)
+    buf = guarded.view
     with qn.qn_create(n, m, g.dtype) as h:
         qn.qn_gram(h, g, buf)
         torch.cuda.synchronize()
         assert h.last_launches == 2
+    guarded.check()
     C = buf[: m * m].view(m, m).cpu().numpy()
     w = buf[m * m:].cpu().numpy()
     Cref = oracle.gram(W.to_bits(g))
@@ -256,7 +201,8 @@ def test_async_window_matches_sync_oracle(qn, dtype, m, n, writes):
     """Config 3's protocol at reduced n: fill the window, then single-Worker Writes each replacing the oldest
     column with an update after each; every update is compared with the oracle run on the window's contents."""
     cfg = W.Config(3, n, m, dtype, -2, 2, 0, 0.1, 1e-3, 1.0, 0.01, writes=writes)
-    out = torch.empty(n, dtype=cfg.torch_dtype, device="cuda")
+    guarded = Guarded(n, cfg.torch_dtype)
+    out = guarded.view
     win_t = np.zeros((m, n), dtype=np.float32 if dtype == "f32" else np.uint16)
     win_g = np.zeros_like(win_t)
     with qn.qn_create(n, m, cfg.torch_dtype) as h:
@@ -277,6 +223,10 @@ def test_async_window_matches_sync_oracle(qn, dtype, m, n, writes):
                 assert np.max(np.abs(np.array(sigma) - ref.sigma)) <= 1e-5 * ref.sigma[0]
                 got = oracle.storage_to_f64(W.to_bits(out))
                 assert np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL[dtype]
+        guarded.check()
+        # every Write landed in its own slot and touched no other row of the window
+        dev_t, dev_g = window_bits(qn, h, cfg.torch_dtype)
+        assert np.array_equal(dev_t, win_t) and np.array_equal(dev_g, win_g)
         # incremental Gram == full recomputation from the window
         j1, s1, _ = qn.qn_update_window(h, cfg.tau, cfg.lam, out)
         a = out.clone()
@@ -383,10 +333,12 @@ def test_apply_hinv_matches_the_oracle(qn, dtype, m, n):
     z = torch.randn(n, device="cuda", generator=gen).to(theta.dtype)
     # a z with a large part inside span{u_k}: a combination of the gradients themselves
     z = (z.float() + 0.5 * (g[1].float() - g[0].float()) - 0.25 * (g[m - 1].float() - g[2].float())).to(theta.dtype)
-    out = torch.empty(n, dtype=theta.dtype, device="cuda")
+    guarded = Guarded(n, theta.dtype)
+    out = guarded.view
     with qn.qn_create(n, m, theta.dtype) as h:
         j, sigma, status = qn.qn_apply_hinv(h, theta, g, cfg.lam, z, out)
         assert h.last_launches == 4
+    guarded.check()
     ref, jref = oracle.apply_hinv(W.to_bits(theta), W.to_bits(g), cfg.lam, oracle.storage_to_f64(W.to_bits(z)))
     assert status == 0 and j == jref and 0 < j < m - 1
     got = oracle.storage_to_f64(W.to_bits(out))
@@ -558,9 +510,6 @@ def test_direct_gram_reference_by_lambda(qn, m, lam):
 def test_tensor_core_gram_path(qn, dtype, m, n, gap):
     """Above 2^22 columns and 8 Workers the Gram pass runs on the tensor cores (bf16 hi/lo split, fp32
     accumulation in short chains).  Same bar as everywhere: exact j, sigma and theta_new tolerances."""
-    import os
-
-    assert os.environ.get("QN_GRAM_PATH", "") != "alu"
     cfg = W.Config(40, n, m, dtype, -2, 2, 0, 0.01, 1e-4, 1.0, 0.01)
     lam = 0.05 if (gap and dtype == "bf16") else 0.01
     theta, g = W.generate(cfg, "cuda", gap_lam=lam if gap else None, gap_scale=1.0 if (gap and dtype == "bf16") else None)
@@ -569,20 +518,19 @@ def test_tensor_core_gram_path(qn, dtype, m, n, gap):
 
 
 def test_tensor_core_and_alu_paths_agree(qn):
-    """The same input through the tensor-core kernel and (QN_GRAM_PATH=alu) the plain-ALU kernel."""
-    import os
-
+    """The same input through the tensor-core kernel and (qn_set_gram_path) the plain-ALU kernel."""
     cfg = W.Config(41, 1 << 22, 24, "f32", -2, 2, 0, 0.01, 1e-4, 1.0, 0.01)
     theta, g = W.generate(cfg, "cuda", gap_lam=0.01)
-    out = {}
-    for path in ("tc", "alu"):
-        os.environ["QN_GRAM_PATH"] = path
-        try:
-            out[path] = run_gpu(qn, theta, g, cfg.tau, cfg.lam)
-        finally:
-            os.environ.pop("QN_GRAM_PATH", None)
-    (o1, j1, s1, st1, _), (o2, j2, s2, st2, _) = out["tc"], out["alu"]
+    res = {}
+    for path in (qn.QN_GRAM_PATH_AUTO, qn.QN_GRAM_PATH_PLAIN_ALU):
+        out = torch.empty(cfg.n, dtype=theta.dtype, device="cuda")
+        with qn.qn_create(cfg.n, cfg.m, theta.dtype) as h:
+            qn.qn_set_gram_path(h, path)
+            j, sigma, status = qn.qn_update(h, theta, g, cfg.tau, cfg.lam, out)
+        res[path] = (out, j, np.array(sigma), status)
+    (o1, j1, s1, st1), (o2, j2, s2, st2) = res[qn.QN_GRAM_PATH_AUTO], res[qn.QN_GRAM_PATH_PLAIN_ALU]
     assert st1 == 0 and st2 == 0 and j1 == j2
+    assert not np.array_equal(s1, s2)  # two different kernels ran
     assert np.max(np.abs(s1[:j1] - s2[:j1]) / s2[:j1]) <= 1e-5
     assert torch.linalg.norm(o1.double() - o2.double()) / torch.linalg.norm(o2.double()) <= 1e-5
 
@@ -595,77 +543,150 @@ def test_tensor_core_path_bitwise_reproducible(qn):
     assert ja == jb and np.array_equal(sa, sb) and torch.equal(a.view(torch.int32), b.view(torch.int32))
 
 
-# --------------------------------------------------------------------------- full size, in the benchmark's launch configuration
-def test_config2_full_size_sampled(qn):
-    """Config 2 at its full n = 25.6 M, m = 32, fp32, exactly as bench.py launches it: j and sigma from the
-    oracle's full passes over the same bits, theta_new on 4096 sampled columns (first, last, tile edges, random)."""
-    cfg = W.CONFIGS[2]
-    theta, g = W.generate(cfg, "cuda")
-    rng = np.random.default_rng(7)
-    idx = np.unique(np.concatenate([[0, 1, 63, 64, 127, 128, cfg.n - 1, cfg.n - 64, cfg.n - 65],
-                                    rng.integers(0, cfg.n, 4096)])).astype(np.int64)
-    rel, j, _ = check_against_oracle(qn, theta, g, cfg.tau, cfg.lam, cfg.dtype, expect_j=cfg.m - 1, sample=idx)
-    assert j == cfg.m - 1
+# --------------------------------------------------------------------------- tensor-core path on structured data
+@pytest.mark.parametrize("lam", [1e-2])
+@pytest.mark.parametrize("kind", ["repeated", "one_worker"])
+def test_tensor_core_gram_on_structured_residuals(qn, kind, lam):
+    """fp32 storage, m = 32, n = 2^22 on the tensor-core path at the configurations' lambda, with inputs on which rounding errors cannot be
+    assumed to average out like independent ones: (repeated) the Workers' deviations take 64 column patterns and
+    the common part 4 values, so every rounding error of the 16-bit split recurs n / 256 times; (one_worker) the
+    largest mode of the spectrum sits on one Worker, the small retained modes on the others.  Same bar."""
+    m, n = 32, 1 << 22
+    if kind == "repeated":
+        theta, g = W.repeated_patterns(n, m, "f32", lam, "cuda")
+    else:
+        cfg = W.Config(47, n, m, "f32", -2, 2, 0, 0.01, 1e-4, 1.0, lam)
+        theta, g = W.generate(cfg, "cuda", gap_lam=lam, gap_scale=1.0, top_on_one_worker=True)
+    expect = assert_gap(theta, g, lam)
+    assert 2 < expect < m - 1
+    check_against_oracle(qn, theta, g, 1.0, lam, "f32", expect_j=expect)
 
 
-def test_config3_full_size_sampled(qn):
-    """Config 3 at its full n = 124 M, m = 8, bf16, as bench.py launches it: the window is filled, then two
-    single-Worker Writes replace the oldest columns (bulk-copy row refresh), with an update after the fill and
-    after each Write.  j and sigma from the oracle's full passes over the window's bits, theta_new on sampled
-    columns."""
-    cfg = W.CONFIGS[3]
+# --------------------------------------------------------------------------- restore, sweep limit, pointer checks
+def test_window_restore_from_saved_columns(qn):
+    """Resume path of the asynchronous mode: allocate the window, copy saved (theta, g) columns into its storage,
+    mark it full, rebuild the raw Gram, update -- equal to the oracle on those columns; then one more Write on top."""
+    cfg = W.Config(3, 50_008, 6, "bf16", -2, 2, 0, 0.1, 1e-3, 1.0, 0.01)
     n, m = cfg.n, cfg.m
-    out = torch.empty(n, dtype=cfg.torch_dtype, device="cuda")
-    win_t = np.zeros((m, n), dtype=np.uint16)
-    win_g = np.zeros_like(win_t)
-    rng = np.random.default_rng(11)
-    idx = np.unique(np.concatenate([[0, 1, 7, 8, 2047, 2048, n - 1, n - 8, n - 9], rng.integers(0, n, 4096)])).astype(np.int64)
+    cols = [W.write_column(cfg, t, "cuda") for t in range(m + 1)]
+    saved_t = torch.stack([c[0] for c in cols[:m]]).contiguous()
+    saved_g = torch.stack([c[1] for c in cols[:m]]).contiguous()
+    guarded = Guarded(n, cfg.torch_dtype)
+    out = guarded.view
     with qn.qn_create(n, m, cfg.torch_dtype) as h:
-        for t in range(m + 2):
-            th, gr = W.write_column(cfg, t, "cuda")
-            slot = t % m
-            qn.qn_push(h, -1, th, gr)
-            win_t[slot], win_g[slot] = W.to_bits(th), W.to_bits(gr)
-            del th, gr
-            if t < m - 1:
-                continue
-            j, sigma, status = qn.qn_update_window(h, cfg.tau, cfg.lam, out)
-            assert h.last_launches == 2
-            if t in (m - 1, m + 1):
-                ref = oracle.update(win_t, win_g, cfg.tau, cfg.lam, sample_idx=idx)
-                assert status == 0 and j == ref.j == m - 1
-                assert np.max(np.abs(np.array(sigma) - ref.sigma)) <= 1e-5 * ref.sigma[0]
-                assert np.max(np.abs(np.array(sigma)[:j] - ref.sigma[:j]) / ref.sigma[:j]) <= 1e-5
-                got = oracle.storage_to_f64(W.to_bits(out))[idx]
-                assert np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL["bf16"]
+        assert qn.qn_window_ptrs(h) == (0, 0)
+        qn.qn_window_alloc(h)
+        pt, pg = qn.qn_window_ptrs(h)
+        assert pt and pg
+        with pytest.raises(qn.QNError) as e:  # allocated but not filled
+            qn.qn_update_window(h, cfg.tau, cfg.lam, out)
+        assert e.value.status == qn.QN_ERR_STATE
+        copy_device_bytes(pt, saved_t.data_ptr(), saved_t.numel() * 2)
+        copy_device_bytes(pg, saved_g.data_ptr(), saved_g.numel() * 2)
+        qn.qn_window_mark_full(h)
+        qn.qn_rebuild(h)
+        j, sigma, status = qn.qn_update_window(h, cfg.tau, cfg.lam, out)
+        ref = oracle.update(W.to_bits(saved_t), W.to_bits(saved_g), cfg.tau, cfg.lam)
+        assert status == 0 and j == ref.j
+        assert np.max(np.abs(np.array(sigma) - ref.sigma)) <= 1e-5 * ref.sigma[0]
+        got = oracle.storage_to_f64(W.to_bits(out))
+        assert np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL["bf16"]
+        # a Write after the restore replaces slot 0 (the restored window's oldest pair)
+        qn.qn_push(h, -1, *cols[m])
+        j, sigma, status = qn.qn_update_window(h, cfg.tau, cfg.lam, out)
+        wt, wg = W.to_bits(saved_t).copy(), W.to_bits(saved_g).copy()
+        wt[0], wg[0] = W.to_bits(cols[m][0]), W.to_bits(cols[m][1])
+        ref = oracle.update(wt, wg, cfg.tau, cfg.lam)
+        assert status == 0 and j == ref.j
+        got = oracle.storage_to_f64(W.to_bits(out))
+        assert np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL["bf16"]
+        dev_t, dev_g = window_bits(qn, h, cfg.torch_dtype)
+        assert np.array_equal(dev_t, wt) and np.array_equal(dev_g, wg)
+    guarded.check()
 
 
-@pytest.mark.parametrize("m", W.CONFIG4_M_SWEEP)
-def test_config4_full_size_by_tiling(qn, m):
-    """Config 4 at its full n = 2^28, bf16, at every m of its sweep as bench.py launches it (m = 64: 68.7 GB of
-    inputs) is beyond what the oracle can read in a test.  Property used instead: if the columns repeat with period p, the Gram is (n/p) times the block's Gram,
-    so sigma scales by sqrt(n/p), j is unchanged and theta_new repeats with the block's values.  The block
-    (p = 2^18 columns) goes through the oracle; the full-size input goes through the library."""
-    free, _ = torch.cuda.mem_get_info()
-    cfg = W.CONFIGS[4].with_shape(m=m)
-    need = 2 * cfg.m * cfg.n * 2 + cfg.n * 2 + (2 << 30)
-    if free < need:
-        pytest.skip("needs %.0f GB of free device memory" % (need / 1e9))
-    p = 1 << 18
-    block = cfg.with_shape(n=p)
-    tb, gb = W.generate(block, "cuda")
-    theta = W.tile_columns(tb, cfg.n)
-    g = W.tile_columns(gb, cfg.n)
-    out, j, sigma, status, launches = run_gpu(qn, theta, g, cfg.tau, cfg.lam)
-    del theta, g
-    ref = oracle.update(W.to_bits(tb), W.to_bits(gb), cfg.tau, cfg.lam)
-    assert status == 0 and launches == 3 and j == ref.j == cfg.m - 1
-    scale = np.sqrt(cfg.n / p)
-    assert np.max(np.abs(sigma - scale * ref.sigma)) <= 1e-5 * scale * ref.sigma[0]
-    assert np.max(np.abs(sigma[:j] - scale * ref.sigma[:j]) / (scale * ref.sigma[:j])) <= 1e-5
-    got = oracle.storage_to_f64(W.to_bits(out))
-    for start in (0, p, 7 * p, cfg.n - p):
-        seg = got[start:start + p]
-        assert np.linalg.norm(seg - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL["bf16"]
-    # every period holds the same bits
-    assert torch.equal(out[:p].view(torch.int16), out[cfg.n - p:].view(torch.int16))
+def test_sweep_limit_reports_not_converged_and_still_writes(qn):
+    """With the Jacobi sweeps capped at one the eigen-solve cannot finish: the step reports QN_ERR_NOT_CONVERGED,
+    theta_new, j and sigma are still written (from the matrix as it stands), and lifting the cap restores the
+    converged result.  qn_last_sweeps follows."""
+    cfg = W.Config(48, 20_000, 8, "f32", -1, 1, 0, 0.1, 1e-3, 0.7, 0.02)
+    theta, g = W.generate(cfg, "cuda", gap_lam=cfg.lam, gap_scale=1.0)
+    ref = oracle.update(W.to_bits(theta), W.to_bits(g), cfg.tau, cfg.lam)
+    out = torch.full((cfg.n,), float("nan"), dtype=torch.float32, device="cuda")
+    with qn.qn_create(cfg.n, cfg.m, torch.float32) as h:
+        assert h.last_sweeps == -1
+        qn.qn_set_sweep_limit(h, 1)
+        j, sigma, status = qn.qn_update(h, theta, g, cfg.tau, cfg.lam, out)
+        assert status == qn.QN_ERR_NOT_CONVERGED and h.last_sweeps == 1
+        assert bool(torch.isfinite(out).all()) and np.all(np.isfinite(sigma)) and 0 <= j <= cfg.m - 1
+        assert qn.qn_status_sync(h) == qn.QN_ERR_NOT_CONVERGED
+        qn.qn_set_sweep_limit(h, None)
+        j, sigma, status = qn.qn_update(h, theta, g, cfg.tau, cfg.lam, out)
+        assert status == 0 and j == ref.j and 2 <= h.last_sweeps <= 12
+        got = oracle.storage_to_f64(W.to_bits(out))
+        assert np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL["f32"]
+    with pytest.raises(qn.QNError):
+        qn.qn_set_sweep_limit(qn.Handle(0, 1, 1, torch.float32), 1)
+
+
+def test_pointers_that_the_device_cannot_read_are_refused(qn):
+    """A host pointer where a device pointer belongs is refused before any launch (it would fault on the device)."""
+    import ctypes
+
+    L = qn.lib()
+    n, m = 1000, 4
+    t = torch.zeros(m, n, device="cuda")
+    o = torch.zeros(n, device="cuda")
+    host = torch.zeros(m, n)
+    host_o = torch.zeros(n)
+    gram = torch.zeros(m * m + m, dtype=torch.float64, device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+    with qn.qn_create(n, m, torch.float32) as h:
+        tp, op, hp, hop = t.data_ptr(), o.data_ptr(), host.data_ptr(), host_o.data_ptr()
+        assert L.qn_update(h.ptr, hp, tp, 1.0, 0.1, op, None, None, st) == qn.QN_ERR_INVALID
+        assert L.qn_update(h.ptr, tp, hp, 1.0, 0.1, op, None, None, st) == qn.QN_ERR_INVALID
+        assert L.qn_update(h.ptr, tp, tp, 1.0, 0.1, hop, None, None, st) == qn.QN_ERR_INVALID
+        assert L.qn_gram(h.ptr, hp, gram.data_ptr(), st) == qn.QN_ERR_INVALID
+        assert L.qn_update_from_gram(h.ptr, tp, tp, host.data_ptr(), 1.0, 0.1, op, None, None, st) == qn.QN_ERR_INVALID
+        assert L.qn_push(h.ptr, -1, hop, op, st) == qn.QN_ERR_INVALID
+        assert L.qn_update(h.ptr, tp, tp, 1.0, 0.1, op, None, None, st) == qn.QN_OK
+        assert qn.qn_status_sync(h) in (qn.QN_OK, qn.QN_ERR_NONFINITE)
+        assert h.total_launches == 3  # only the accepted call launched anything
+
+
+# --------------------------------------------------------------------------- n-sharded step as a program
+def test_sharded_step_inside_a_process_group(qn):
+    """qn_update_sharded itself, inside an initialised one-rank NCCL process group and on a stream that is not
+    torch's current one: Gram pass, all-reduce (the identity for one rank, but it runs, on the stream the kernels
+    use) and the step from the reduced buffer, with and without host results; equal to the oracle."""
+    import torch.distributed as dist
+
+    from test_multi_rank_cpu import _free_port
+
+    cfg = W.Config(49, (1 << 22) + 64, 32, "f32", -1, 1, 0, 0.1, 1e-3, 0.7, 0.02)
+    theta, g = W.generate(cfg, "cuda", gap_lam=cfg.lam, gap_scale=1.0)
+    ref = oracle.update(W.to_bits(theta), W.to_bits(g), cfg.tau, cfg.lam)
+    created = not dist.is_initialized()
+    if created:
+        dist.init_process_group("nccl", init_method="tcp://127.0.0.1:%d" % _free_port(), rank=0, world_size=1,
+                                device_id=torch.device("cuda", torch.cuda.current_device()))
+    try:
+        side = torch.cuda.Stream()
+        buf = torch.empty(cfg.m * cfg.m + cfg.m, dtype=torch.float64, device="cuda")
+        out = torch.empty(cfg.n, dtype=theta.dtype, device="cuda")
+        torch.cuda.synchronize()
+        with qn.qn_create(cfg.n, cfg.m, theta.dtype) as h:
+            j, sigma, status = qn.qn_update_sharded(h, theta, g, cfg.tau, cfg.lam, out, buf, stream=side)
+            assert h.last_launches == 2 and h.total_launches == 4
+            assert status == 0 and j == ref.j
+            assert np.max(np.abs(np.array(sigma) - ref.sigma)) <= 1e-5 * ref.sigma[0]
+            got = oracle.storage_to_f64(W.to_bits(out))
+            assert np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL["f32"]
+            first = out.clone()
+            out.zero_()
+            assert qn.qn_update_sharded(h, theta, g, cfg.tau, cfg.lam, out, buf, want_host=False, stream=side) is None
+            side.synchronize()
+            assert torch.equal(out, first)
+    finally:
+        if created:
+            dist.destroy_process_group()

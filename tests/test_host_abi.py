@@ -54,6 +54,47 @@ def test_null_handle_is_rejected(qn):
     assert L.qn_rebuild(None, None) == qn.QN_ERR_INVALID
     assert L.qn_status_sync(None) == qn.QN_ERR_INVALID
     assert L.qn_last_launches(None) == 0
+    assert L.qn_set_sweep_limit(None, 3) == qn.QN_ERR_INVALID
+    assert L.qn_set_gram_path(None, 0) == qn.QN_ERR_INVALID
+
+
+class _FakeCudaTensor:
+    """Stands in for a CUDA tensor on a machine without one: the binding's checks read only these attributes."""
+
+    def __init__(self, shape, dtype, index):
+        self.shape, self.dtype, self.is_cuda = shape, dtype, True
+        self.device = torch.device("cuda", index)
+
+    def is_contiguous(self):
+        return True
+
+    def numel(self):
+        n = 1
+        for s in self.shape:
+            n *= s
+        return n
+
+    def data_ptr(self):
+        raise AssertionError("a tensor on the wrong device must be refused before its pointer is taken")
+
+
+def test_binding_refuses_tensors_of_another_device(qn):
+    """A tensor on another GPU than the handle's would make the kernels dereference memory they cannot reach (a
+    device fault, not an error code), so the binding refuses it on the host."""
+    h = qn.Handle(0, 100, 4, torch.float32, device=1)
+    with pytest.raises(ValueError, match="cuda:0"):
+        qn._dev_matrix(_FakeCudaTensor((4, 100), torch.float32, 0), h, "theta")
+    with pytest.raises(ValueError, match="cuda:3"):
+        qn._dev_vector(_FakeCudaTensor((100,), torch.float32, 3), h, "theta_new")
+    with pytest.raises(ValueError, match="cuda:0"):
+        qn._check_gram_buffer(h, _FakeCudaTensor((20,), torch.float64, 0))
+    with pytest.raises(ValueError, match="same device"):
+        g = _FakeCudaTensor((4, 100), torch.float32, 0)
+        g.dim = lambda: 2
+        qn.qn_gram_static(g, _FakeCudaTensor((20,), torch.float64, 1))
+    # the same objects on the handle's device pass the device check and reach data_ptr()
+    with pytest.raises(AssertionError):
+        qn._dev_matrix(_FakeCudaTensor((4, 100), torch.float32, 1), h, "theta")
 
 
 @pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-device behaviour")

@@ -121,22 +121,28 @@ def gap_spectrum(m: int, lam: float) -> torch.Tensor:
     return torch.tensor(np.sort(s)[::-1].copy(), dtype=torch.float64)
 
 
-def _perturbation(cfg: Config, device, c: int, cols: int, gap_lam: Optional[float], gap_scale: float) -> torch.Tensor:
+def _perturbation(cfg: Config, device, c: int, cols: int, gap_lam: Optional[float], gap_scale: float,
+                  top_on_one_worker: bool = False) -> torch.Tensor:
     """theta_k - theta0 on one chunk, [m][cols] fp32.
 
     Literal recipe: iid N(0, pert^2).  Gap variant: Z diag(s) Q^T with Z iid N(0,1), Q the Helmert
     basis and s = ``gap_spectrum`` -- the singular values of the centred matrices then follow s, which
-    leaves a gap around lam * sigma_1 so that the cut-off j is well defined."""
+    leaves a gap around lam * sigma_1 so that the cut-off j is well defined.  The Helmert basis puts the
+    largest mode on Workers 0 and 1; ``top_on_one_worker`` reverses the spectrum's order along the basis,
+    so that the largest mode is carried by the last Worker alone (against the mean of the others)."""
     if gap_lam is None:
         return cfg.pert * _normal((cfg.m, cols), device, _gen(device, cfg.seed, _S_PERT, c))
     Z = _normal((cfg.m - 1, cols), device, _gen(device, cfg.seed, _S_Z, c)).double()
     s = gap_spectrum(cfg.m, gap_lam).to(device)
+    if top_on_one_worker:
+        s = torch.flip(s, dims=(0,))
     Q = helmert(cfg.m, device)
     return (gap_scale * (Q * s) @ Z).float()
 
 
 def generate(cfg: Config, device="cpu", gap_lam: Optional[float] = None, gap_scale: Optional[float] = None,
-             out: Optional[Tuple[torch.Tensor, torch.Tensor]] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+             out: Optional[Tuple[torch.Tensor, torch.Tensor]] = None,
+             top_on_one_worker: bool = False) -> Tuple[torch.Tensor, torch.Tensor]:
     """theta[m][n], g[m][n] in the config's storage dtype on ``device``.
 
     g_k = D theta_k + W (W^T theta_k) - b + noise, computed in fp32 from the unrounded theta_k, then
@@ -155,12 +161,12 @@ def generate(cfg: Config, device="cpu", gap_lam: Optional[float] = None, gap_sca
         wt = torch.zeros((cfg.rank, m), dtype=torch.float64, device=device)
         for c, i0, i1 in _chunks(n):
             _, _, theta0 = _problem_chunk(cfg, device, c, i1 - i0)
-            th = theta0.unsqueeze(0) + _perturbation(cfg, device, c, i1 - i0, gap_lam, scale)
+            th = theta0.unsqueeze(0) + _perturbation(cfg, device, c, i1 - i0, gap_lam, scale, top_on_one_worker)
             wt += (_w_chunk(cfg, device, c, i1 - i0).double() @ th.double().t())
     for c, i0, i1 in _chunks(n):
         cols = i1 - i0
         D, b, theta0 = _problem_chunk(cfg, device, c, cols)
-        th = theta0.unsqueeze(0) + _perturbation(cfg, device, c, cols, gap_lam, scale)
+        th = theta0.unsqueeze(0) + _perturbation(cfg, device, c, cols, gap_lam, scale, top_on_one_worker)
         gr = D.unsqueeze(0) * th - b.unsqueeze(0)
         if wt is not None:
             gr += (wt.t().float() @ _w_chunk(cfg, device, c, cols))
@@ -234,3 +240,58 @@ def tile_columns(block: torch.Tensor, n: int) -> torch.Tensor:
     if block.dim() == 1:
         return block.repeat(reps)[:n].contiguous()
     return block.repeat(1, reps)[:, :n].contiguous()
+
+
+def period_permutation(p: int, q: int, seed: int, device="cpu") -> torch.Tensor:
+    """The column permutation of period q of ``tile_columns_permuted`` (int64, length p)."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed((seed * 2_654_435_761 + q * 40_503 + 17) % (1 << 62))
+    return torch.randperm(p, generator=gen).to(device)
+
+
+def tile_columns_permuted(block: torch.Tensor, n: int, seed: int) -> torch.Tensor:
+    """Like ``tile_columns``, but every period holds its own seeded permutation of the block's columns:
+    column q*p + c of the result is column ``period_permutation(p, q, seed)[c]`` of the block.  Any quantity that
+    is a sum over columns is still (n/p) times the block's, while a result per column can be traced back to its
+    source column, so a column offset that is a multiple of p no longer goes unnoticed."""
+    p = block.shape[-1]
+    if n % p:
+        raise ValueError("n must be a multiple of the block's width")
+    out = torch.empty(block.shape[:-1] + (n,), dtype=block.dtype, device=block.device)
+    for q in range(n // p):
+        out[..., q * p:(q + 1) * p] = block.index_select(-1, period_permutation(p, q, seed, block.device))
+    return out
+
+
+def repeated_patterns(n: int, m: int, dtype: str, lam: float, device="cpu", scale: float = 0.25,
+                      patterns: int = 64, bases=(0.75, -1.25, 2.5, 0.3125)) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Inputs whose columns repeat a small set of values, for checks of reduced-precision Gram arithmetic.
+
+    The Workers' deviations take only ``patterns`` distinct column patterns, X_P = scale * (Q diag(s)) Z_P with Q the
+    Helmert basis, s = ``gap_spectrum(m, lam)`` and Z_P the rows 1..m-1 of the Sylvester Hadamard matrix of order
+    ``patterns`` (entries +-1, orthogonal rows, so the singular values follow s exactly); the common part of a column
+    takes the ``len(bases)`` values of ``bases`` in turn.  g_k[i] = bases[i % B] + X_P[k][(i // B) % patterns] and
+    theta_k[i] = theta0[i] + X_P[k][..] / 2, rounded to the storage dtype.  Every rounding error of a kernel that
+    splits or truncates the deviations is therefore repeated n / (B * patterns) times instead of averaging out over
+    the n columns."""
+    if patterns & (patterns - 1) or patterns < m:
+        raise ValueError("patterns must be a power of two >= m")
+    device = torch.device(device)
+    idx = torch.arange(patterns, dtype=torch.int64)
+    had = torch.tensor([[1.0 - 2.0 * (bin(r & c).count("1") & 1) for c in range(patterns)] for r in range(1, m)],
+                       dtype=torch.float64)
+    s = gap_spectrum(m, lam)
+    XP = (scale * (helmert(m) * s) @ had).to(device)                 # [m][patterns], fp64
+    B = len(bases)
+    base = torch.tensor(bases, dtype=torch.float64, device=device)
+    tdtype = torch.float32 if dtype == "f32" else torch.bfloat16
+    theta = torch.empty((m, n), dtype=tdtype, device=device)
+    g = torch.empty((m, n), dtype=tdtype, device=device)
+    for c, i0, i1 in _chunks(n):
+        i = torch.arange(i0, i1, dtype=torch.int64, device=device)
+        x = XP[:, (i // B) % patterns]
+        theta0 = _normal(i1 - i0, device, _gen(device, BASE_SEED + 99, _S_THETA0, c)).double()
+        g[:, i0:i1] = (base[i % B].unsqueeze(0) + x).float().to(tdtype)
+        theta[:, i0:i1] = (theta0.unsqueeze(0) + 0.5 * x).float().to(tdtype)
+    del idx
+    return theta, g
