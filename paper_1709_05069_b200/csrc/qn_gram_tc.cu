@@ -102,6 +102,12 @@ constexpr int kTcRunBytes = QN_TC_RUN_BYTES;           // bytes of one row that 
 #ifndef QN_TC_FASTPATH_F32
 #define QN_TC_FASTPATH_F32 1
 #endif
+#ifndef QN_TC_CHAIN_F32
+#define QN_TC_CHAIN_F32 2
+#endif
+#ifndef QN_TC_CHAIN_BF16
+#define QN_TC_CHAIN_BF16 4
+#endif
 
 template <typename T, int MP>
 struct TcShape {
@@ -130,7 +136,7 @@ struct TcShape {
     static_assert(kStagesPerItem <= kTcRelease, "the stages of an item belong to one release group");
     // Stages per accumulation chain = per drain.  The error of a chain grows with its length; bf16 storage
     // (hi + lo exact, no input rounding at all) has the margin for 16 instructions, fp32 storage keeps 8.
-    static constexpr int kChainStages = sizeof(T) == 2 ? 4 : 2;
+    static constexpr int kChainStages = sizeof(T) == 2 ? QN_TC_CHAIN_BF16 : QN_TC_CHAIN_F32;
     static_assert(kStages % kTcRelease == 0 && kChainStages % kTcRelease == 0, "whole release groups");
     static_assert(kTeams * kStagesPerItem <= 2 * kStages * kItemsPerStage, "a warp's consecutive items are at most two revolutions apart");
 };
