@@ -259,6 +259,22 @@ QN_API qn_status qn_selftest_bounded_wait(qn_handle h, void* cuda_stream);
 QN_API int32_t qn_last_launches(qn_handle h);
 QN_API int64_t qn_total_launches(qn_handle h);
 
+/*
+ * Which kernel the most recent Gram pass of this handle was dispatched to (qn_update, qn_update_host, qn_gram,
+ * qn_apply_hinv, qn_rebuild), or, after qn_push, which row-refresh kernel ran; QN_KERNEL_NONE before the first.
+ * Benchmarks label their numbers with it.  QN_KERNEL_FP64_PRODUCTS is or-ed in when every product and sum of the
+ * pass was formed in fp64 (n below 2^22, and qn_rebuild).
+ */
+#define QN_KERNEL_NONE 0
+#define QN_KERNEL_GRAM_DIRECT 1  /* m <= 8, register-fed, plain ALUs */
+#define QN_KERNEL_GRAM_BULK 2    /* m <= 8, fed by bulk copies into shared-memory stages, packed fp32 ALUs */
+#define QN_KERNEL_GRAM_TILED 3   /* 9 <= m <= 64, shared-memory tiles, plain ALUs */
+#define QN_KERNEL_GRAM_TENSOR 4  /* 9 <= m <= 64, tcgen05 tensor cores, bf16 hi/lo split, fp32 chains, fp64 flush */
+#define QN_KERNEL_ROW_REGISTER 5 /* row refresh, register-fed */
+#define QN_KERNEL_ROW_BULK 6     /* row refresh, fed and landed by bulk copies */
+#define QN_KERNEL_FP64_PRODUCTS 0x100
+QN_API int32_t qn_last_gram_kernel(qn_handle h);
+
 /* Jacobi sweeps used by the most recent step whose results were fetched to the host (j_out or
  * sigma_out non-NULL, or qn_status_sync), else -1. */
 QN_API int32_t qn_last_sweeps(qn_handle h);

@@ -54,6 +54,7 @@ struct qn_ctx {
     int32_t last_launches;
     int64_t total_launches;
     int32_t last_sweeps;
+    int32_t last_kernel;  // QN_KERNEL_* of the most recent Gram or row pass
 };
 
 static int g_sm_count_cache[64];
@@ -170,7 +171,7 @@ qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, do
     {
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st,
-                           &h->last_launches, h->error_word, lambda, h->plain_alu != 0) != cudaSuccess)
+                           &h->last_launches, h->error_word, lambda, h->plain_alu != 0, &h->last_kernel) != cudaSuccess)
             return QN_ERR_CUDA;
     }
     int np_theta = 0;
@@ -182,7 +183,7 @@ qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, do
         }
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, theta, h->n, h->m, false, h->partials_theta, &np_theta, h->max_partials, st,
-                           &h->last_launches, h->error_word, lambda, h->plain_alu != 0) != cudaSuccess)
+                           &h->last_launches, h->error_word, lambda, h->plain_alu != 0, &h->last_kernel) != cudaSuccess)
             return QN_ERR_CUDA;
     }
     qn_solve_params p;
@@ -444,7 +445,7 @@ extern "C" qn_status qn_apply_hinv(qn_handle h, const void* theta, const void* g
     if (s == QN_OK) {
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st, &h->last_launches,
-                           h->error_word, lambda, h->plain_alu != 0) != cudaSuccess)
+                           h->error_word, lambda, h->plain_alu != 0, &h->last_kernel) != cudaSuccess)
             s = QN_ERR_CUDA;
     }
     if (s == QN_OK) {
@@ -488,7 +489,7 @@ extern "C" qn_status qn_gram(qn_handle h, const void* g, double* gram_out, void*
     {
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st, &h->last_launches,
-                           h->error_word, 0.0, h->plain_alu != 0) != cudaSuccess)
+                           h->error_word, 0.0, h->plain_alu != 0, &h->last_kernel) != cudaSuccess)
             s = QN_ERR_CUDA;
     }
     if (s == QN_OK) {
@@ -559,6 +560,8 @@ extern "C" qn_status qn_push(qn_handle h, int32_t slot, const void* theta_col, c
         cudaMemcpyAsync(trow, theta_col, col_bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
         s = QN_ERR_CUDA;
     if (s == QN_OK) {
+        h->last_kernel = (theta_landed ? QN_KERNEL_ROW_BULK : QN_KERNEL_ROW_REGISTER) |
+                         (h->n < QN_PRECISE_BELOW ? QN_KERNEL_FP64_PRODUCTS : 0);
         h->filled |= (1ull << slot);
         if (oldest) h->head = (h->head + 1) % h->m;  // a Write that could not be enqueued does not use up its slot
     }
@@ -618,7 +621,7 @@ extern "C" qn_status qn_rebuild(qn_handle h, void* cuda_stream) {
     int np = 0;
     qn_status s = QN_OK;
     if (qn_launch_gram(h->dtype, h->win_g, h->n, h->m, true, h->partials, &np, h->max_partials, st,
-                       &h->last_launches) != cudaSuccess)
+                       &h->last_launches, nullptr, 0.0, false, &h->last_kernel) != cudaSuccess)
         s = QN_ERR_CUDA;
     if (s == QN_OK) {
         qn_solve_params p;
@@ -709,6 +712,7 @@ extern "C" qn_status qn_selftest_bounded_wait(qn_handle h, void* cuda_stream) {
 extern "C" int32_t qn_last_launches(qn_handle h) { return h ? h->last_launches : 0; }
 extern "C" int64_t qn_total_launches(qn_handle h) { return h ? h->total_launches : 0; }
 extern "C" int32_t qn_last_sweeps(qn_handle h) { return h ? h->last_sweeps : -1; }
+extern "C" int32_t qn_last_gram_kernel(qn_handle h) { return h ? h->last_kernel : QN_KERNEL_NONE; }
 
 extern "C" qn_status qn_timing_begin(qn_handle h, int32_t max_kernels) {
     if (!h || max_kernels < 1 || max_kernels > (1 << 20)) return QN_ERR_INVALID;

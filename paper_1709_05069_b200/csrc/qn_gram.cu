@@ -733,26 +733,32 @@ static cudaError_t launch_gram_t(const T* g, int64_t n, int m, bool raw, double*
 
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
                            int* num_partials, int max_partials, cudaStream_t st, int* launches, int* error_word,
-                           double lambda_hint, bool plain_alu) {
+                           double lambda_hint, bool plain_alu, int* kernel_out) {
     cudaError_t e;
     const int64_t elem = dtype == QN_F32 ? 4 : 2;
+    int kernel;
     if (!raw && !plain_alu && qn_gram_tc_applicable(dtype, g, n, m)) {
+        kernel = QN_KERNEL_GRAM_TENSOR;
         e = qn_launch_gram_tc(dtype, g, n, m, partials, num_partials, max_partials, error_word, st);
     } else if (!raw && !plain_alu && m <= qn::kDirectM && n >= QN_PRECISE_BELOW &&
                reinterpret_cast<uintptr_t>(g) % 16 == 0 && (n * elem) % 16 == 0) {
         // bulk-copy variant of the direct kernel (plain_alu keeps the register-fed one, for A/B runs)
         const bool ref0 = lambda_hint >= QN_REF0_MIN_LAMBDA;
+        kernel = QN_KERNEL_GRAM_BULK;
         e = dtype == QN_F32 ? qn::launch_gram_stream(static_cast<const float*>(g), n, m, partials, num_partials,
                                                      max_partials, error_word, false, st)
                             : qn::launch_gram_stream(static_cast<const __nv_bfloat16*>(g), n, m, partials,
                                                      num_partials, max_partials, error_word, ref0, st);
     } else {
+        kernel = (m <= qn::kDirectM ? QN_KERNEL_GRAM_DIRECT : QN_KERNEL_GRAM_TILED) |
+                 (raw || n < QN_PRECISE_BELOW ? QN_KERNEL_FP64_PRODUCTS : 0);
         e = dtype == QN_F32
                 ? qn::launch_gram_t(static_cast<const float*>(g), n, m, raw, partials, num_partials, max_partials, st)
                 : qn::launch_gram_t(static_cast<const __nv_bfloat16*>(g), n, m, raw, partials, num_partials,
                                     max_partials, st);
     }
     if (e == cudaSuccess && launches) *launches += 1;
+    if (e == cudaSuccess && kernel_out) *kernel_out = kernel;
     return e;
 }
 

@@ -80,7 +80,8 @@ struct qn_solve_params {
 // plain_alu: keep to the register-fed plain-ALU kernels (qn_set_gram_path; A/B measurements and tests).
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
                            int* num_partials, int max_partials, cudaStream_t st, int* launches,
-                           int* error_word = nullptr, double lambda_hint = 0.0, bool plain_alu = false);
+                           int* error_word = nullptr, double lambda_hint = 0.0, bool plain_alu = false,
+                           int* kernel_out = nullptr);  // kernel_out: which kernel was dispatched (QN_KERNEL_* of qn.h)
 // Loads every Gram kernel variant into the current context (allocates nothing the caller can see later: after it,
 // the first launch of a variant no longer loads code).
 cudaError_t qn_gram_preload();

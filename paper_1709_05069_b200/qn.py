@@ -28,10 +28,20 @@ EXPORTS = (
     "qn_set_rank_cap", "qn_set_sweep_limit", "qn_set_gram_path", "qn_set_tau_cap", "qn_last_tau", "qn_push",
     "qn_update_window", "qn_rebuild",
     "qn_window_alloc", "qn_window_theta", "qn_window_g", "qn_window_mark_full", "qn_update_host", "qn_status_sync",
-    "qn_last_launches", "qn_total_launches", "qn_last_sweeps", "qn_timing_begin", "qn_timing_end",
+    "qn_last_launches", "qn_total_launches", "qn_last_sweeps", "qn_last_gram_kernel", "qn_timing_begin",
+    "qn_timing_end",
     "qn_gram_static", "qn_selftest_bounded_wait",
 )
 TIME_KINDS = ("gram", "solve", "combine", "row")
+KERNEL_NAMES = {
+    0: "none",
+    1: "direct (m <= 8, register-fed, plain ALUs)",
+    2: "bulk-copy (m <= 8, shared-memory stages, packed fp32 ALUs, fp64 flush)",
+    3: "tiled (plain ALUs)",
+    4: "tcgen05 (bf16 hi/lo split, fp32 accumulation in short chains, fp64 flush)",
+    5: "row refresh, register-fed",
+    6: "row refresh, bulk-copy (fp32 sums per work item, fp64 across)",
+}
 
 
 class QNError(RuntimeError):
@@ -74,6 +84,7 @@ def lib() -> ctypes.CDLL:
         L.qn_last_launches.argtypes, L.qn_last_launches.restype = [vp], i32
         L.qn_total_launches.argtypes, L.qn_total_launches.restype = [vp], i64
         L.qn_last_sweeps.argtypes, L.qn_last_sweeps.restype = [vp], i32
+        L.qn_last_gram_kernel.argtypes, L.qn_last_gram_kernel.restype = [vp], i32
         L.qn_gram_static.argtypes, L.qn_gram_static.restype = [i64, i32, i32, vp, vp, vp], i32
         L.qn_timing_begin.argtypes, L.qn_timing_begin.restype = [vp, i32], i32
         L.qn_timing_end.argtypes, L.qn_timing_end.restype = [vp, vp, vp], i32
@@ -134,6 +145,13 @@ class Handle:
     @property
     def last_sweeps(self) -> int:
         return lib().qn_last_sweeps(self.ptr)
+
+    @property
+    def last_gram_kernel(self) -> str:
+        """Name of the kernel the most recent Gram pass (or row refresh) was dispatched to."""
+        code = lib().qn_last_gram_kernel(self.ptr)
+        name = KERNEL_NAMES.get(code & 0xff, "unknown")
+        return name + (", fp64 products and sums" if code & 0x100 else "")
 
 
 def _stream_ptr(stream) -> int:

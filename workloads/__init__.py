@@ -176,6 +176,54 @@ def generate(cfg: Config, device="cpu", gap_lam: Optional[float] = None, gap_sca
     return theta, g
 
 
+def low_rank_products(cfg: Config, device, begin: int, end: int, gap_lam: Optional[float] = None,
+                      gap_scale: Optional[float] = None) -> Optional[torch.Tensor]:
+    """The part of W^T theta_k (r x m, fp64) that the columns [begin, end) contribute, or None for a diagonal A.
+    ``begin`` and ``end`` must be multiples of the generation chunk (or ``end`` = n).  Summed over a partition of
+    [0, n) in chunk order this is what ``generate`` forms in its first pass; a process that holds only a slice of
+    the columns adds these over the processes before it calls ``generate_slice``."""
+    if cfg.rank == 0:
+        return None
+    device = torch.device(device)
+    scale = cfg.pert if gap_scale is None else gap_scale
+    wt = torch.zeros((cfg.rank, cfg.m), dtype=torch.float64, device=device)
+    for c, i0, i1 in _chunks(cfg.n):
+        if i1 <= begin or i0 >= end:
+            continue
+        if i0 < begin or i1 > end:
+            raise ValueError("slice boundaries must fall on generation chunks")
+        _, _, theta0 = _problem_chunk(cfg, device, c, i1 - i0)
+        th = theta0.unsqueeze(0) + _perturbation(cfg, device, c, i1 - i0, gap_lam, scale)
+        wt += (_w_chunk(cfg, device, c, i1 - i0).double() @ th.double().t())
+    return wt
+
+
+def generate_slice(cfg: Config, device, begin: int, end: int, wt: Optional[torch.Tensor],
+                   gap_lam: Optional[float] = None, gap_scale: Optional[float] = None):
+    """Columns [begin, end) of what ``generate(cfg)`` returns, as theta[m][end-begin], g[m][end-begin], without
+    forming the rest: for a process that holds one slice of an n-sharded problem.  ``wt`` is the full W^T theta
+    (``low_rank_products`` added over all slices; None for a diagonal A)."""
+    device = torch.device(device)
+    m = cfg.m
+    scale = cfg.pert if gap_scale is None else gap_scale
+    theta = torch.empty((m, end - begin), dtype=cfg.torch_dtype, device=device)
+    g = torch.empty((m, end - begin), dtype=cfg.torch_dtype, device=device)
+    for c, i0, i1 in _chunks(cfg.n):
+        if i1 <= begin or i0 >= end:
+            continue
+        cols = i1 - i0
+        D, b, theta0 = _problem_chunk(cfg, device, c, cols)
+        th = theta0.unsqueeze(0) + _perturbation(cfg, device, c, cols, gap_lam, scale)
+        gr = D.unsqueeze(0) * th - b.unsqueeze(0)
+        if wt is not None:
+            gr += (wt.t().float() @ _w_chunk(cfg, device, c, cols))
+        gr += cfg.noise * _normal((m, cols), device, _gen(device, cfg.seed, _S_NOISE, c))
+        lo, hi = max(i0, begin), min(i1, end)
+        theta[:, lo - begin:hi - begin] = th[:, lo - i0:hi - i0].to(cfg.torch_dtype)
+        g[:, lo - begin:hi - begin] = gr[:, lo - i0:hi - i0].to(cfg.torch_dtype)
+    return theta, g
+
+
 def write_column(cfg: Config, t: int, device="cpu") -> Tuple[torch.Tensor, torch.Tensor]:
     """The (theta, g) pair of the t-th asynchronous single-Worker Write, each [n] in storage dtype.
 
