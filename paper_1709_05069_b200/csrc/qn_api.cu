@@ -55,6 +55,7 @@ struct qn_ctx {
     int64_t total_launches;
     int32_t last_sweeps;
     int32_t last_kernel;  // QN_KERNEL_* of the most recent Gram or row pass
+    int32_t redo_kernel;  // QN_KERNEL_* of the fp64 repeat pass that the most recent step enqueued (0: none)
 };
 
 static int g_sm_count_cache[64];
@@ -137,6 +138,7 @@ qn_status fetch_result(qn_handle h, cudaStream_t st, int32_t* j_out, double* sig
     if (sigma_out) memcpy(sigma_out, h->host_result->sigma, sizeof(double) * h->m);
     h->last_sweeps = h->host_result->sweeps;
     h->last_tau = h->host_result->tau_eff;
+    if ((h->host_result->redo & 2) && h->redo_kernel) h->last_kernel = h->redo_kernel;  // the fp64 repeat pass ran
     return static_cast<qn_status>(h->host_result->status);
 }
 
@@ -163,6 +165,30 @@ bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
     return a0 < b0 + nb && b0 < a0 + na;
 }
 
+// After the first solve of a step whose Gram pass had reduced precision: the same pass with every product in fp64,
+// and a second solve.  Both kernels return at once unless the first solve found a retained sigma_k so small that the
+// reduced-precision pass cannot deliver it to 1e-5 (result->redo, on the device: the host does not wait to find out).
+qn_status precise_redo(qn_handle h, const void* g, qn_solve_params p, double lambda, cudaStream_t st) {
+    h->redo_kernel = 0;
+    p.redo_coeff = qn_gram_error_coeff(h->last_kernel, h->dtype, h->n, lambda);
+    if (!(p.redo_coeff > 0.0)) return QN_OK;
+    // every retained sigma_k is at least lambda sigma_1: with this lambda the first solve cannot ask for a repeat
+    if (lambda >= 1.0 || p.redo_coeff / (lambda * lambda) <= QN_REDO_TRIGGER) return QN_OK;
+    const int* run_if = &h->result->redo;  // device address; not dereferenced here
+    int np = 0;
+    {
+        KernelTimer t(h, st, QN_TIME_GRAM);
+        if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st, &h->last_launches,
+                           h->error_word, lambda, true, &h->redo_kernel, run_if) != cudaSuccess)
+            return QN_ERR_CUDA;
+    }
+    p.num_partials = np;
+    p.only_if_redo = 1;
+    p.redo_coeff = 0.0;
+    KernelTimer t(h, st, QN_TIME_SOLVE);
+    return qn_launch_solve(p, st, &h->last_launches) == cudaSuccess ? QN_OK : QN_ERR_CUDA;
+}
+
 // Gram partials -> solve -> combine on device buffers.
 // theta_ready (may be NULL): an event the stream waits for before the first kernel that reads theta.
 qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, double lambda, void* theta_new,
@@ -183,7 +209,7 @@ qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, do
         }
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, theta, h->n, h->m, false, h->partials_theta, &np_theta, h->max_partials, st,
-                           &h->last_launches, h->error_word, lambda, h->plain_alu != 0, &h->last_kernel) != cudaSuccess)
+                           &h->last_launches, h->error_word, lambda, h->plain_alu != 0) != cudaSuccess)
             return QN_ERR_CUDA;
     }
     qn_solve_params p;
@@ -202,10 +228,12 @@ qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, do
     p.coef = h->coef;
     p.result = h->result;
     p.error_word = h->error_word;
+    p.redo_coeff = qn_gram_error_coeff(h->last_kernel, h->dtype, h->n, lambda);
     {
         KernelTimer t(h, st, QN_TIME_SOLVE);
         if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) return QN_ERR_CUDA;
     }
+    if (precise_redo(h, g, p, lambda, st) != QN_OK) return QN_ERR_CUDA;
     if (theta_ready && cudaStreamWaitEvent(st, theta_ready, 0) != cudaSuccess) return QN_ERR_CUDA;
     {
         KernelTimer t(h, st, QN_TIME_COMBINE);
@@ -463,8 +491,12 @@ extern "C" qn_status qn_apply_hinv(qn_handle h, const void* theta, const void* g
         p.coef = h->coef;
         p.result = h->result;
         p.error_word = h->error_word;
-        KernelTimer t(h, st, QN_TIME_SOLVE);
-        if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) s = QN_ERR_CUDA;
+        p.redo_coeff = qn_gram_error_coeff(h->last_kernel, h->dtype, h->n, lambda);
+        {
+            KernelTimer t(h, st, QN_TIME_SOLVE);
+            if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) s = QN_ERR_CUDA;
+        }
+        if (s == QN_OK) s = precise_redo(h, g, p, lambda, st);
     }
     if (s == QN_OK) {
         KernelTimer t(h, st, QN_TIME_COMBINE);

@@ -17,6 +17,8 @@
 //             carry the cancellation of the later m x m centring.
 // Every thread owns fixed columns and fixed output entries, so results are bitwise reproducible for
 // a given grid.
+#include <math.h>
+
 #include "qn_device.cuh"
 
 namespace qn {
@@ -96,7 +98,8 @@ struct DirectItem {
 
 template <typename T, bool kAligned, int kMode>
 __global__ void __launch_bounds__(kThreads, 1)
-gram_direct_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ partials) {
+gram_direct_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ partials, const int* __restrict__ run_if) {
+    if (run_if && (*run_if & 1) == 0) return;  // a repeat pass that the spectrum did not ask for
     using Item = DirectItem<T, kAligned>;
     constexpr int kCols = Item::kCols;
     constexpr int kFlushIters = kFlushCols / kCols > 0 ? kFlushCols / kCols : 1;
@@ -466,7 +469,8 @@ struct TiledSmem {
 
 template <typename T, bool kAligned, int kMode>
 __global__ void __launch_bounds__(kThreads, 1)
-gram_tiled_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ partials) {
+gram_tiled_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict__ partials, const int* __restrict__ run_if) {
+    if (run_if && (*run_if & 1) == 0) return;  // a repeat pass that the spectrum did not ask for
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TiledSmem& sm = *reinterpret_cast<TiledSmem*>(smem_raw);
 
@@ -690,22 +694,23 @@ gram_tiled_kernel(const T* __restrict__ g, int64_t n, int m, double* __restrict_
 // Host side
 // ------------------------------------------------------------------------------------------------
 template <typename T, bool kAligned, int kMode>
-static cudaError_t launch_gram_mode(const T* g, int64_t n, int m, double* partials, int grid, cudaStream_t st) {
+static cudaError_t launch_gram_mode(const T* g, int64_t n, int m, double* partials, int grid, cudaStream_t st,
+                                    const int* run_if) {
     if (m <= kDirectM) {
-        gram_direct_kernel<T, kAligned, kMode><<<grid, kThreads, 0, st>>>(g, n, m, partials);
+        gram_direct_kernel<T, kAligned, kMode><<<grid, kThreads, 0, st>>>(g, n, m, partials, run_if);
         return cudaGetLastError();
     }
     auto kern = gram_tiled_kernel<T, kAligned, kMode>;
     const size_t smem = sizeof(TiledSmem);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kern<<<grid, kThreads, smem, st>>>(g, n, m, partials);
+    kern<<<grid, kThreads, smem, st>>>(g, n, m, partials, run_if);
     return cudaGetLastError();
 }
 
 template <typename T>
 static cudaError_t launch_gram_t(const T* g, int64_t n, int m, bool raw, double* partials, int* num_partials,
-                                 int max_partials, cudaStream_t st) {
+                                 int max_partials, cudaStream_t st, const int* run_if = nullptr) {
     const bool aligned = (reinterpret_cast<uintptr_t>(g) % 16 == 0) && ((n * (int64_t)sizeof(T)) % 16 == 0);
     const int sms = qn_sm_count();
     int64_t ntiles;
@@ -718,26 +723,32 @@ static cudaError_t launch_gram_t(const T* g, int64_t n, int m, bool raw, double*
     int grid = (int)(ntiles < sms ? ntiles : sms);
     if (grid > max_partials) grid = max_partials;
     *num_partials = grid;
-    const int mode = raw ? kRaw : (n < QN_PRECISE_BELOW ? kPrecise : kFast);
+    const int mode = raw ? kRaw : (n < QN_PRECISE_BELOW || run_if ? kPrecise : kFast);
     if (aligned) {
-        if (mode == kRaw) return launch_gram_mode<T, true, kRaw>(g, n, m, partials, grid, st);
-        if (mode == kPrecise) return launch_gram_mode<T, true, kPrecise>(g, n, m, partials, grid, st);
-        return launch_gram_mode<T, true, kFast>(g, n, m, partials, grid, st);
+        if (mode == kRaw) return launch_gram_mode<T, true, kRaw>(g, n, m, partials, grid, st, run_if);
+        if (mode == kPrecise) return launch_gram_mode<T, true, kPrecise>(g, n, m, partials, grid, st, run_if);
+        return launch_gram_mode<T, true, kFast>(g, n, m, partials, grid, st, run_if);
     }
-    if (mode == kRaw) return launch_gram_mode<T, false, kRaw>(g, n, m, partials, grid, st);
-    if (mode == kPrecise) return launch_gram_mode<T, false, kPrecise>(g, n, m, partials, grid, st);
-    return launch_gram_mode<T, false, kFast>(g, n, m, partials, grid, st);
+    if (mode == kRaw) return launch_gram_mode<T, false, kRaw>(g, n, m, partials, grid, st, run_if);
+    if (mode == kPrecise) return launch_gram_mode<T, false, kPrecise>(g, n, m, partials, grid, st, run_if);
+    return launch_gram_mode<T, false, kFast>(g, n, m, partials, grid, st, run_if);
 }
 
 }  // namespace qn
 
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
                            int* num_partials, int max_partials, cudaStream_t st, int* launches, int* error_word,
-                           double lambda_hint, bool plain_alu, int* kernel_out) {
+                           double lambda_hint, bool plain_alu, int* kernel_out, const int* run_if) {
     cudaError_t e;
     const int64_t elem = dtype == QN_F32 ? 4 : 2;
     int kernel;
-    if (!raw && !plain_alu && qn_gram_tc_applicable(dtype, g, n, m)) {
+    if (run_if) {
+        kernel = (m <= qn::kDirectM ? QN_KERNEL_GRAM_DIRECT : QN_KERNEL_GRAM_TILED) | QN_KERNEL_FP64_PRODUCTS;
+        e = dtype == QN_F32 ? qn::launch_gram_t(static_cast<const float*>(g), n, m, false, partials, num_partials,
+                                                max_partials, st, run_if)
+                            : qn::launch_gram_t(static_cast<const __nv_bfloat16*>(g), n, m, false, partials,
+                                                num_partials, max_partials, st, run_if);
+    } else if (!raw && !plain_alu && qn_gram_tc_applicable(dtype, g, n, m)) {
         kernel = QN_KERNEL_GRAM_TENSOR;
         e = qn_launch_gram_tc(dtype, g, n, m, partials, num_partials, max_partials, error_word, st);
     } else if (!raw && !plain_alu && m <= qn::kDirectM && n >= QN_PRECISE_BELOW &&
@@ -760,6 +771,19 @@ cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool
     if (e == cudaSuccess && launches) *launches += 1;
     if (e == cudaSuccess && kernel_out) *kernel_out = kernel;
     return e;
+}
+
+double qn_gram_error_coeff(int kernel, qn_dtype dtype, int64_t n, double lambda_hint) {
+    if (kernel & QN_KERNEL_FP64_PRODUCTS) return 0.0;
+    const double by_n = sqrt((double)QN_PRECISE_BELOW / (double)(n > QN_PRECISE_BELOW ? n : QN_PRECISE_BELOW));
+    switch (kernel & 0xff) {
+        case QN_KERNEL_GRAM_TENSOR: return dtype == QN_F32 ? QN_REDO_COEFF_TC_F32 : QN_REDO_COEFF_TC_BF16;
+        case QN_KERNEL_GRAM_BULK:
+            return (dtype == QN_BF16 && lambda_hint >= QN_REF0_MIN_LAMBDA ? QN_REDO_COEFF_REF0_AT_4M : QN_REDO_COEFF_ALU_AT_4M) * by_n;
+        case QN_KERNEL_GRAM_DIRECT:
+        case QN_KERNEL_GRAM_TILED: return QN_REDO_COEFF_ALU_AT_4M * by_n;
+    }
+    return 0.0;
 }
 
 namespace qn {

@@ -27,7 +27,8 @@ struct qn_result_block {
     int32_t j;
     int32_t status;  // qn_status seen on the device (OK, NOT_CONVERGED, NONFINITE)
     int32_t sweeps;
-    int32_t pad;
+    int32_t redo;    // bit 0: the spectrum asks for the Gram pass to be repeated in fp64 (set by the first solve, cleared
+                     // by the second); bit 1: the results come from such a repeated pass
     double sigma[QN_MAX_M];
     double tau_eff;  // the learning rate the step used (tau, or less under the learning-rate cap)
 };
@@ -66,6 +67,10 @@ struct qn_solve_params {
     int32_t num_partials_theta;
     const double* rhs_raw;  // NULL, or m doubles g_k^T z: the coefficients are then built for z instead of gbar
                             // (w = P rhs_raw) and with tau = -1, i.e. for out = z - G d + Theta d (Eq. (4))
+    double redo_coeff;    // > 0: the Gram came from a reduced-precision pass whose relative error on a retained sigma_k is
+                          // about redo_coeff * (sigma_1 / sigma_k)^2; if that exceeds QN_REDO_TRIGGER for the smallest
+                          // retained one, result->redo bit 0 is set (the step then repeats the pass in fp64)
+    int32_t only_if_redo; // != 0: return at once unless result->redo bit 0 is set (the second solve of such a step)
     qn_coef_block* coef;
     qn_result_block* result;
     int* error_word;      // device int set by a kernel that gave up on a bounded wait (may be NULL); read and cleared
@@ -77,11 +82,27 @@ struct qn_solve_params {
 // bulk-copy kernel for bf16 storage and m <= 8 may take Worker 0 instead of the mean as its per-column reference
 // (a third fewer instructions; the error of a retained sigma_k grows as 1 / lambda^2, see qn_gram.cu).
 #define QN_REF0_MIN_LAMBDA 0.01
+// Predicted relative error of the smallest retained sigma above which the Gram pass is repeated in fp64 (a quarter
+// of the 1e-5 the library promises), and the measured error coefficients of the reduced-precision passes (relative
+// error of sigma_k = coefficient * (sigma_1 / sigma_k)^2 on inputs whose largest modes sit on few Workers):
+//   tensor cores: the fp32 accumulator truncates each product, a bias proportional to the chain length and
+//                 independent of n: 2e-9 for fp32 storage (chains of 8 instructions), 2e-8 for bf16 (16)
+//   fp32 products on the plain ALUs: unbiased, 2e-10 at n = 2^22 and falling as 1 / sqrt(n); the bulk-copy kernel
+//                 with Worker 0 as its reference 2e-9 at n = 2^22
+#define QN_REDO_TRIGGER 2.5e-6
+#define QN_REDO_COEFF_TC_F32 2e-9
+#define QN_REDO_COEFF_TC_BF16 2e-8
+#define QN_REDO_COEFF_ALU_AT_4M 2e-10
+#define QN_REDO_COEFF_REF0_AT_4M 2e-9
 // plain_alu: keep to the register-fed plain-ALU kernels (qn_set_gram_path; A/B measurements and tests).
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
                            int* num_partials, int max_partials, cudaStream_t st, int* launches,
                            int* error_word = nullptr, double lambda_hint = 0.0, bool plain_alu = false,
-                           int* kernel_out = nullptr);  // kernel_out: which kernel was dispatched (QN_KERNEL_* of qn.h)
+                           int* kernel_out = nullptr,  // kernel_out: which kernel was dispatched (QN_KERNEL_* of qn.h)
+                           const int* run_if = nullptr);  // run_if: the pass forms every product in fp64 on the plain
+                                                          // ALUs and returns at once unless bit 0 of *run_if is set
+// Error coefficient (see QN_REDO_TRIGGER) of the pass that `kernel` (QN_KERNEL_*) stands for; 0 for an fp64 pass.
+double qn_gram_error_coeff(int kernel, qn_dtype dtype, int64_t n, double lambda_hint);
 // Loads every Gram kernel variant into the current context (allocates nothing the caller can see later: after it,
 // the first launch of a variant no longer loads code).
 cudaError_t qn_gram_preload();

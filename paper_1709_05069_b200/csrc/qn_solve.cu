@@ -169,6 +169,8 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
     const int m = prm.m;
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int tri_len = m * (m + 1) / 2;
+    // the second solve of a step whose Gram pass was repeated in fp64: nothing to do unless the first one asked for it
+    if (prm.only_if_redo && (prm.result->redo & 1) == 0) return;
 
     if (tid == 0) {
         sm.flag_nonfinite = 0;
@@ -259,6 +261,7 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
             prm.result->status = sm.flag_timeout ? QN_ERR_DEVICE_TIMEOUT : sm.flag_nonfinite ? QN_ERR_NONFINITE : QN_OK;
             prm.result->j = 0;
             prm.result->sweeps = 0;
+            prm.result->redo = 0;
         }
         return;
     }
@@ -274,6 +277,7 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
             prm.result->j = 0;
             prm.result->status = sm.flag_timeout ? QN_ERR_DEVICE_TIMEOUT : QN_ERR_NONFINITE;
             prm.result->sweeps = 0;
+            prm.result->redo = prm.only_if_redo ? 2 : 0;
             prm.result->tau_eff = prm.tau;
         }
         return;
@@ -574,6 +578,15 @@ __global__ void __launch_bounds__(1024, 1) solve_kernel(qn_solve_params prm) {
         prm.result->j = j;
         prm.result->status = sm.flag_timeout ? QN_ERR_DEVICE_TIMEOUT : converged ? QN_OK : QN_ERR_NOT_CONVERGED;
         prm.result->sweeps = sweeps;
+        // A reduced-precision Gram pass leaves an error of about redo_coeff * (sigma_1 / sigma_k)^2 on sigma_k: if
+        // that is too much for the smallest retained one, ask for the pass to be repeated in fp64 (the sigma computed
+        // here are good enough to decide: the trigger sits a factor of four below what the library promises).
+        int redo = prm.only_if_redo ? 2 : 0;
+        if (prm.redo_coeff > 0.0 && j > 0 && sm.sigma[j - 1] > 0.0) {
+            const double ratio = sm.sigma[0] / sm.sigma[j - 1];
+            if (prm.redo_coeff * ratio * ratio > QN_REDO_TRIGGER) redo = 1;
+        }
+        prm.result->redo = redo;
     }
 }
 

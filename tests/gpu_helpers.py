@@ -36,8 +36,16 @@ def run_gpu(qn, theta, g, tau, lam):
     with qn.qn_create(n, m, theta.dtype) as h:
         j, sigma, status = qn.qn_update(h, theta, g, tau, lam, out)
         launches = h.last_launches
+        run_gpu.last_kernel = h.last_gram_kernel  # which Gram kernel delivered the result
     guarded.check()
     return out, j, np.array(sigma), status, launches
+
+
+def step_launches(n, base=3):
+    """Kernels of one step: from 2^22 parameters on the Gram pass has reduced precision, and unless lambda is so
+    large that no retained mode can need it, the step enqueues a conditional fp64 repeat of the pass and of the solve
+    (both return at once unless the spectrum asks for them)."""
+    return (base,) if n < (1 << 22) else (base, base + 2)
 
 
 def _cudart():
@@ -73,7 +81,7 @@ def check_against_oracle(qn, theta, g, tau, lam, dtype, expect_j=None, sample=No
     tb, gb = W.to_bits(theta), W.to_bits(g)
     ref = oracle.update(tb, gb, tau, lam, sample_idx=sample)
     assert status == 0
-    assert launches == 3
+    assert launches in step_launches(theta.shape[1])
     assert j == ref.j, (j, ref.j, sigma / sigma[0], ref.sigma / ref.sigma[0])
     if expect_j is not None:
         assert j == expect_j

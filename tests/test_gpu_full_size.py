@@ -182,7 +182,7 @@ def test_config4_full_size_by_permuted_tiling(qn, m):
     out, j, sigma, status, launches = run_gpu(qn, theta, g, cfg.tau, cfg.lam)
     del theta, g
     ref = oracle.update(W.to_bits(tb), W.to_bits(gb), cfg.tau, cfg.lam)
-    assert status == 0 and launches == 3 and j == ref.j == cfg.m - 1
+    assert status == 0 and launches in (3, 5) and j == ref.j == cfg.m - 1
     scale = np.sqrt(cfg.n / p)
     assert np.max(np.abs(sigma - scale * ref.sigma)) <= 1e-5 * scale * ref.sigma[0]
     assert np.max(np.abs(sigma[:j] - scale * ref.sigma[:j]) / (scale * ref.sigma[:j])) <= 1e-5
