@@ -104,10 +104,17 @@ QN_API qn_status qn_destroy(qn_handle h);
  * relative 1e-5; theta_new within a relative L2 error of 1e-5 (fp32 storage) or 2e-3 (bf16 storage: the single
  * rounding of the output).  The arithmetic of the Gram pass is chosen from n, m, the storage type and lambda
  * (fp64 products below 2^22 parameters; fp32 or tensor-core products above), never from the data.
- * Condition on the sigma figures above 2^22 parameters: there the products are rounded (fp32, or for m > 8 and
- * fp32 storage the 16 leading bits of each centred value on the tensor cores), and the bound relies on these
- * rounding errors adding up like independent ones over the n columns (error of a retained sigma_k about
- * 1e-5 sigma_1 / sqrt(n) per unit of 1 / lambda).  qn_set_gram_path(QN_GRAM_PATH_PLAIN_ALU) keeps fp32 products.
+ * How the sigma figures are kept above 2^22 parameters.  There the Gram pass rounds: fp32 products on the plain ALUs
+ * (unbiased; the relative error of a retained sigma_k is about 2e-10 (sigma_1 / sigma_k)^2 at n = 2^22 and falls as
+ * 1 / sqrt(n)), or for m > 8 the tensor cores, whose fp32 accumulator truncates each product: measured, a retained
+ * sigma_k comes out low by about 2e-9 (fp32 storage) or 2e-8 (bf16 storage) times (sigma_1 / sigma_k)^2, whatever n.
+ * Whether that is within the promise depends on the spectrum, so it is checked on the device: the eigen-solve compares
+ * the smallest retained sigma_k with the pass's error coefficient (a factor of four inside 1e-5), and where it falls
+ * short the Gram pass is repeated with every product in fp64 and the solve re-run, before the pass that writes
+ * theta_new; nothing waits on the host.  A step therefore launches three kernels, or five of which two return at once
+ * (when lambda is so small that some spectrum could need the repeat), and costs two to ten times more on inputs that do
+ * need it.  qn_update, qn_update_host and qn_apply_hinv work this way; qn_gram and qn_update_from_gram do not see the
+ * spectrum before the caller's reduction (see QN_GRAM_PATH_FP64), and the asynchronous window forms fp32 products.
  */
 QN_API qn_status qn_update(qn_handle h, const void* theta, const void* g, double tau, double lambda,
                     void* theta_new, int32_t* j_out, double* sigma_out, void* cuda_stream);
@@ -135,10 +142,14 @@ QN_API qn_status qn_set_sweep_limit(qn_handle h, int32_t max_sweeps);
  *   QN_GRAM_PATH_AUTO       the default: tensor-core kernel for m > 8, bulk-copy kernel for m <= 8, both from
  *                           2^22 parameters on aligned rows; the register-fed plain-ALU kernels elsewhere
  *   QN_GRAM_PATH_PLAIN_ALU  the register-fed plain-ALU kernels everywhere (same results within the stated accuracy)
+ *   QN_GRAM_PATH_FP64       the plain-ALU kernels with every product and sum in fp64 whatever n (several times slower
+ *                           than the others above 2^22 parameters): for qn_gram / qn_update_from_gram callers whose
+ *                           spectrum has retained modes far below sigma_1 (see the accuracy notes of those calls)
  * Host-side setting of the handle; nothing is read from the environment.
  */
 #define QN_GRAM_PATH_AUTO 0
 #define QN_GRAM_PATH_PLAIN_ALU 1
+#define QN_GRAM_PATH_FP64 2
 QN_API qn_status qn_set_gram_path(qn_handle h, int32_t path);
 
 /*

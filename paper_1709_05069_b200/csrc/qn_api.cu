@@ -26,7 +26,7 @@ struct qn_ctx {
     double* rhs;                  // device, m doubles: g_k^T z of qn_apply_hinv
     int32_t j_cap;                // < 0: none
     int32_t sweep_limit;          // limit on the fp64 Jacobi sweeps, 0 = the built-in one
-    int32_t plain_alu;            // Gram pass restricted to the plain-ALU kernels (qn_set_gram_path)
+    int32_t gram_path;            // QN_GRAM_PATH_* (qn_set_gram_path)
     int32_t tau_cap;              // learning-rate cap on/off (qn_update and qn_update_host)
     double* partials_theta;       // device, as `partials`, allocated when the cap is first switched on
     double last_tau;              // learning rate of the most recent step whose results were fetched
@@ -179,7 +179,7 @@ qn_status precise_redo(qn_handle h, const void* g, qn_solve_params p, double lam
     {
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st, &h->last_launches,
-                           h->error_word, lambda, true, &h->redo_kernel, run_if) != cudaSuccess)
+                           h->error_word, lambda, QN_GRAM_PATH_FP64, &h->redo_kernel, run_if) != cudaSuccess)
             return QN_ERR_CUDA;
     }
     p.num_partials = np;
@@ -197,7 +197,7 @@ qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, do
     {
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st,
-                           &h->last_launches, h->error_word, lambda, h->plain_alu != 0, &h->last_kernel) != cudaSuccess)
+                           &h->last_launches, h->error_word, lambda, h->gram_path, &h->last_kernel) != cudaSuccess)
             return QN_ERR_CUDA;
     }
     int np_theta = 0;
@@ -209,7 +209,7 @@ qn_status run_step(qn_handle h, const void* theta, const void* g, double tau, do
         }
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, theta, h->n, h->m, false, h->partials_theta, &np_theta, h->max_partials, st,
-                           &h->last_launches, h->error_word, lambda, h->plain_alu != 0) != cudaSuccess)
+                           &h->last_launches, h->error_word, lambda, h->gram_path) != cudaSuccess)
             return QN_ERR_CUDA;
     }
     qn_solve_params p;
@@ -373,8 +373,9 @@ extern "C" qn_status qn_set_sweep_limit(qn_handle h, int32_t max_sweeps) {
 }
 
 extern "C" qn_status qn_set_gram_path(qn_handle h, int32_t path) {
-    if (!h || (path != QN_GRAM_PATH_AUTO && path != QN_GRAM_PATH_PLAIN_ALU)) return QN_ERR_INVALID;
-    h->plain_alu = path == QN_GRAM_PATH_PLAIN_ALU;
+    if (!h || (path != QN_GRAM_PATH_AUTO && path != QN_GRAM_PATH_PLAIN_ALU && path != QN_GRAM_PATH_FP64))
+        return QN_ERR_INVALID;
+    h->gram_path = path;
     return QN_OK;
 }
 
@@ -473,7 +474,7 @@ extern "C" qn_status qn_apply_hinv(qn_handle h, const void* theta, const void* g
     if (s == QN_OK) {
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st, &h->last_launches,
-                           h->error_word, lambda, h->plain_alu != 0, &h->last_kernel) != cudaSuccess)
+                           h->error_word, lambda, h->gram_path, &h->last_kernel) != cudaSuccess)
             s = QN_ERR_CUDA;
     }
     if (s == QN_OK) {
@@ -521,7 +522,7 @@ extern "C" qn_status qn_gram(qn_handle h, const void* g, double* gram_out, void*
     {
         KernelTimer t(h, st, QN_TIME_GRAM);
         if (qn_launch_gram(h->dtype, g, h->n, h->m, false, h->partials, &np, h->max_partials, st, &h->last_launches,
-                           h->error_word, 0.0, h->plain_alu != 0, &h->last_kernel) != cudaSuccess)
+                           h->error_word, 0.0, h->gram_path, &h->last_kernel) != cudaSuccess)
             s = QN_ERR_CUDA;
     }
     if (s == QN_OK) {
@@ -653,7 +654,7 @@ extern "C" qn_status qn_rebuild(qn_handle h, void* cuda_stream) {
     int np = 0;
     qn_status s = QN_OK;
     if (qn_launch_gram(h->dtype, h->win_g, h->n, h->m, true, h->partials, &np, h->max_partials, st,
-                       &h->last_launches, nullptr, 0.0, false, &h->last_kernel) != cudaSuccess)
+                       &h->last_launches, nullptr, 0.0, QN_GRAM_PATH_AUTO, &h->last_kernel) != cudaSuccess)
         s = QN_ERR_CUDA;
     if (s == QN_OK) {
         qn_solve_params p;

@@ -710,7 +710,8 @@ static cudaError_t launch_gram_mode(const T* g, int64_t n, int m, double* partia
 
 template <typename T>
 static cudaError_t launch_gram_t(const T* g, int64_t n, int m, bool raw, double* partials, int* num_partials,
-                                 int max_partials, cudaStream_t st, const int* run_if = nullptr) {
+                                 int max_partials, cudaStream_t st, const int* run_if = nullptr,
+                                 bool fp64_products = false) {
     const bool aligned = (reinterpret_cast<uintptr_t>(g) % 16 == 0) && ((n * (int64_t)sizeof(T)) % 16 == 0);
     const int sms = qn_sm_count();
     int64_t ntiles;
@@ -723,7 +724,7 @@ static cudaError_t launch_gram_t(const T* g, int64_t n, int m, bool raw, double*
     int grid = (int)(ntiles < sms ? ntiles : sms);
     if (grid > max_partials) grid = max_partials;
     *num_partials = grid;
-    const int mode = raw ? kRaw : (n < QN_PRECISE_BELOW || run_if ? kPrecise : kFast);
+    const int mode = raw ? kRaw : (n < QN_PRECISE_BELOW || fp64_products ? kPrecise : kFast);
     if (aligned) {
         if (mode == kRaw) return launch_gram_mode<T, true, kRaw>(g, n, m, partials, grid, st, run_if);
         if (mode == kPrecise) return launch_gram_mode<T, true, kPrecise>(g, n, m, partials, grid, st, run_if);
@@ -738,16 +739,17 @@ static cudaError_t launch_gram_t(const T* g, int64_t n, int m, bool raw, double*
 
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
                            int* num_partials, int max_partials, cudaStream_t st, int* launches, int* error_word,
-                           double lambda_hint, bool plain_alu, int* kernel_out, const int* run_if) {
+                           double lambda_hint, int path, int* kernel_out, const int* run_if) {
+    const bool plain_alu = path != QN_GRAM_PATH_AUTO;
     cudaError_t e;
     const int64_t elem = dtype == QN_F32 ? 4 : 2;
     int kernel;
-    if (run_if) {
+    if (!raw && (run_if || path == QN_GRAM_PATH_FP64)) {
         kernel = (m <= qn::kDirectM ? QN_KERNEL_GRAM_DIRECT : QN_KERNEL_GRAM_TILED) | QN_KERNEL_FP64_PRODUCTS;
         e = dtype == QN_F32 ? qn::launch_gram_t(static_cast<const float*>(g), n, m, false, partials, num_partials,
-                                                max_partials, st, run_if)
+                                                max_partials, st, run_if, true)
                             : qn::launch_gram_t(static_cast<const __nv_bfloat16*>(g), n, m, false, partials,
-                                                num_partials, max_partials, st, run_if);
+                                                num_partials, max_partials, st, run_if, true);
     } else if (!raw && !plain_alu && qn_gram_tc_applicable(dtype, g, n, m)) {
         kernel = QN_KERNEL_GRAM_TENSOR;
         e = qn_launch_gram_tc(dtype, g, n, m, partials, num_partials, max_partials, error_word, st);

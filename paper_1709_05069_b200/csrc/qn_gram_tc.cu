@@ -748,7 +748,7 @@ bool qn_gram_tc_applicable(qn_dtype dtype, const void* g, int64_t n, int m) {
     const int64_t elem = dtype == QN_F32 ? 4 : 2;
     // every 8-column chunk of a row is fetched with one load: 16 bytes (bf16) or 32 bytes (fp32), aligned
     const int64_t chunk = 8 * elem;
-    return m > 8 && m <= QN_MAX_M && n >= QN_PRECISE_BELOW && (reinterpret_cast<uintptr_t>(g) % chunk == 0) &&
+    return m > 8 && m <= QN_MAX_M && n >= QN_TC_MIN_N && (reinterpret_cast<uintptr_t>(g) % chunk == 0) &&
            (n % 8 == 0);
 }
 

@@ -17,6 +17,13 @@ __host__ __device__ inline int qn_partial_len(int m) { return m * (m + 1) / 2 + 
 // the error of an eigenvalue is about 6e-8 * mu_1 / sqrt(n), which only falls under the 1e-10 * mu_1
 // needed for sigma to be good to 1e-5 * sigma_1 on near-null modes once n is a few million.
 #define QN_PRECISE_BELOW (int64_t(1) << 22)
+// The tensor-core Gram pass (m > 8) starts earlier: its error does not depend on n (the truncating accumulation is a
+// bias), a step checks it against the spectrum on the device and repeats the pass in fp64 where needed, and from
+// about a million columns on it is several times faster than the fp64 pass even though a CTA only gets a few dozen
+// stages.
+#ifndef QN_TC_MIN_N
+#define QN_TC_MIN_N (int64_t(1) << 20)
+#endif
 
 // Eigenvalues of the centred Gram below this fraction of the largest diagonal entry of the
 // uncentred (reference-shifted or raw) Gram are rounding noise of the m x m centring and are set to 0.
@@ -94,10 +101,10 @@ struct qn_solve_params {
 #define QN_REDO_COEFF_TC_BF16 2e-8
 #define QN_REDO_COEFF_ALU_AT_4M 2e-10
 #define QN_REDO_COEFF_REF0_AT_4M 2e-9
-// plain_alu: keep to the register-fed plain-ALU kernels (qn_set_gram_path; A/B measurements and tests).
+// path: QN_GRAM_PATH_* of qn.h (qn_set_gram_path).
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
                            int* num_partials, int max_partials, cudaStream_t st, int* launches,
-                           int* error_word = nullptr, double lambda_hint = 0.0, bool plain_alu = false,
+                           int* error_word = nullptr, double lambda_hint = 0.0, int path = QN_GRAM_PATH_AUTO,
                            int* kernel_out = nullptr,  // kernel_out: which kernel was dispatched (QN_KERNEL_* of qn.h)
                            const int* run_if = nullptr);  // run_if: the pass forms every product in fp64 on the plain
                                                           // ALUs and returns at once unless bit 0 of *run_if is set

@@ -16,6 +16,7 @@ QN_BF16 = 1
 QN_MAX_M = 64
 QN_GRAM_PATH_AUTO = 0
 QN_GRAM_PATH_PLAIN_ALU = 1
+QN_GRAM_PATH_FP64 = 2
 
 (QN_OK, QN_ERR_INVALID, QN_ERR_ALLOC, QN_ERR_CUDA, QN_ERR_STATE, QN_ERR_NOT_CONVERGED, QN_ERR_NONFINITE,
  QN_ERR_DEVICE_TIMEOUT) = range(8)
@@ -234,7 +235,8 @@ def qn_set_sweep_limit(h: Handle, max_sweeps: Optional[int]) -> None:
 
 
 def qn_set_gram_path(h: Handle, path: int) -> None:
-    """``QN_GRAM_PATH_AUTO`` (default) or ``QN_GRAM_PATH_PLAIN_ALU`` (register-fed plain-ALU Gram kernels only)."""
+    """``QN_GRAM_PATH_AUTO`` (default), ``QN_GRAM_PATH_PLAIN_ALU`` (register-fed plain-ALU Gram kernels only) or
+    ``QN_GRAM_PATH_FP64`` (those kernels with fp64 products and sums whatever n)."""
     _check(lib().qn_set_gram_path(h.ptr, int(path)), "qn_set_gram_path")
 
 

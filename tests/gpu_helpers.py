@@ -41,11 +41,11 @@ def run_gpu(qn, theta, g, tau, lam):
     return out, j, np.array(sigma), status, launches
 
 
-def step_launches(n, base=3):
-    """Kernels of one step: from 2^22 parameters on the Gram pass has reduced precision, and unless lambda is so
-    large that no retained mode can need it, the step enqueues a conditional fp64 repeat of the pass and of the solve
-    (both return at once unless the spectrum asks for them)."""
-    return (base,) if n < (1 << 22) else (base, base + 2)
+def step_launches(n, base=3, m=64):
+    """Kernels of one step: from 2^22 parameters on (2^20 with more than 8 Workers: tensor cores) the Gram pass has
+    reduced precision, and unless lambda is so large that no retained mode can need it, the step enqueues a
+    conditional fp64 repeat of the pass and of the solve (both return at once unless the spectrum asks for them)."""
+    return (base,) if n < ((1 << 20) if m > 8 else (1 << 22)) else (base, base + 2)
 
 
 def _cudart():
@@ -81,7 +81,7 @@ def check_against_oracle(qn, theta, g, tau, lam, dtype, expect_j=None, sample=No
     tb, gb = W.to_bits(theta), W.to_bits(g)
     ref = oracle.update(tb, gb, tau, lam, sample_idx=sample)
     assert status == 0
-    assert launches in step_launches(theta.shape[1])
+    assert launches in step_launches(theta.shape[1], 3, theta.shape[0])
     assert j == ref.j, (j, ref.j, sigma / sigma[0], ref.sigma / ref.sigma[0])
     if expect_j is not None:
         assert j == expect_j

@@ -712,3 +712,24 @@ def test_sharded_step_inside_a_process_group(qn):
     finally:
         if created:
             dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("dtype,m", [("f32", 32), ("bf16", 12)])
+def test_gram_paths_at_large_n(qn, dtype, m):
+    """qn_gram above 2^22 parameters: the default path (tensor cores: the whole Gram comes out low by a few 1e-7) and
+    QN_GRAM_PATH_FP64 (every product and sum in fp64), both against the oracle's Gram."""
+    n = (1 << 22) + 64
+    cfg = W.Config(52, n, m, dtype, -1, 1, 0, 0.05, 1e-3, 0.5, 0.05)
+    _, g = W.generate(cfg, "cuda")
+    Cref = oracle.gram(W.to_bits(g))
+    scale = np.abs(Cref).max()
+    for path, tol, name in ((qn.QN_GRAM_PATH_AUTO, 2e-6, "tcgen05"), (qn.QN_GRAM_PATH_FP64, 2e-9, "tiled")):
+        guarded = Guarded(m * m + m, torch.float64)
+        with qn.qn_create(n, m, g.dtype) as h:
+            qn.qn_set_gram_path(h, path)
+            qn.qn_gram(h, g, guarded.view)
+            torch.cuda.synchronize()
+            assert h.last_gram_kernel.startswith(name) and ("fp64" in h.last_gram_kernel) == (path == qn.QN_GRAM_PATH_FP64)
+        guarded.check()
+        C = guarded.view[: m * m].view(m, m).cpu().numpy()
+        assert np.max(np.abs(C - Cref)) <= tol * scale, (path, np.max(np.abs(C - Cref)) / scale)
