@@ -15,9 +15,11 @@
  *
  * Layout.  All matrices are Worker-major: theta[m][n] and g[m][n], row k = Worker k, each row
  * contiguous (the transpose of the paper's n x m matrices).  Elements are fp32 or bf16
- * (qn_dtype); all arithmetic is fp32 products with fp64 accumulation for the Gram, fp64 for the
- * m x m eigen-problem and the coefficients, fp32 for the final combination, and one
- * round-to-nearest-even to the storage type when theta_new is written.
+ * (qn_dtype).  Arithmetic: the Gram pass forms fp64 products below 2^22 parameters and fp32 products
+ * (m <= 8) or tensor-core products of a bf16 hi/lo split (m > 8, from 2^20 parameters on) above, always
+ * with fp64 accumulation across work items, and is repeated in fp64 when the spectrum needs it (see
+ * qn_update); the m x m eigen-problem and the coefficients are fp64; the final combination is fp32 with
+ * one round-to-nearest-even to the storage type when theta_new is written.
  *
  * Pointers.  Unless a parameter says HOST, data pointers are DEVICE pointers on the device that
  * was current when the handle was created.  The caller owns every buffer it passes; the library
@@ -38,7 +40,7 @@
  *
  * Errors.  Every call returns a qn_status; nothing throws or aborts.  Arguments are validated on
  * the host before anything is launched.  Conditions only the device can see (a non-finite Gram,
- * the Jacobi sweep limit) are recorded in a device status word that is returned by the next call
+ * the Jacobi sweep limit, a bounded device wait that ran out) are recorded in a device status word that is returned by the next call
  * that synchronises; in both cases theta_new is still written (with j = 0, i.e. the SGD update,
  * for a non-finite Gram).
  *
@@ -102,9 +104,9 @@ QN_API qn_status qn_destroy(qn_handle h);
  * Accuracy against the exact fp64 evaluation of Eq. (2)-(4) on the stored values: j exact when no sigma_k
  * lies within 1e-5 sigma_1 of lambda sigma_1; every sigma_k within 1e-5 sigma_1, the retained ones within a
  * relative 1e-5; theta_new within a relative L2 error of 1e-5 (fp32 storage) or 2e-3 (bf16 storage: the single
- * rounding of the output).  The arithmetic of the Gram pass is chosen from n, m, the storage type and lambda
- * (fp64 products below 2^22 parameters; fp32 or tensor-core products above), never from the data.
- * How the sigma figures are kept above 2^22 parameters.  There the Gram pass rounds: fp32 products on the plain ALUs
+ * rounding of the output).  The first Gram pass is chosen from n, m, the storage type and lambda (fp64 products
+ * below 2^22 parameters, or 2^20 with m > 8; fp32 or tensor-core products above), never from the data.
+ * How the sigma figures are kept where the Gram pass rounds: fp32 products on the plain ALUs
  * (unbiased; the relative error of a retained sigma_k is about 2e-10 (sigma_1 / sigma_k)^2 at n = 2^22 and falls as
  * 1 / sqrt(n)), or for m > 8 the tensor cores, whose fp32 accumulator truncates each product: measured, a retained
  * sigma_k comes out low by about 2e-9 (fp32 storage) or 2e-8 (bf16 storage) times (sigma_1 / sigma_k)^2, whatever n.
