@@ -208,6 +208,9 @@ QN_API qn_status qn_gram(qn_handle h, const void* g, double* gram_out, void* cud
  *      sigma are the same on every rank.
  *   gram         DEVICE, m*m + m doubles as written by qn_gram (or sums of such buffers), read only
  *   other arguments as for qn_update.  Errors as for qn_update.
+ * Accuracy: that of the Gram it is given.  Above 2^22 parameters (2^20 with m > 8) qn_gram rounds its products (see
+ * qn_update); this call checks the spectrum against that pass's accuracy like qn_update does, but cannot repeat
+ * the pass: see qn_precision_flag.
  */
 QN_API qn_status qn_update_from_gram(qn_handle h, const void* theta, const void* g, const double* gram, double tau,
                                      double lambda, void* theta_new, int32_t* j_out, double* sigma_out,
@@ -230,6 +233,10 @@ QN_API qn_status qn_push(qn_handle h, int32_t slot, const void* theta_col, const
 /*
  * The Server step on the window's current contents.  QN_ERR_STATE until every slot has been
  * written at least once.  Outputs as in qn_update.
+ * Accuracy: above 2^22 parameters the row refresh of qn_push adds fp32 products per work item before it goes to
+ * fp64; measured on spectra with small retained modes, a retained sigma_k is off by about 2e-9 (sigma_1 / sigma_k)^2
+ * of its value with bf16 storage and 5e-12 (sigma_1 / sigma_k)^2 with fp32 storage, whatever n: inside 1e-5 down to
+ * sigma_k = 1.4e-2 sigma_1 (bf16) and 1e-3 sigma_1 (fp32).  qn_rebuild recomputes the window's Gram with fp64 products.
  */
 QN_API qn_status qn_update_window(qn_handle h, double tau, double lambda, void* theta_new, int32_t* j_out,
                            double* sigma_out, void* cuda_stream);
@@ -287,6 +294,16 @@ QN_API int64_t qn_total_launches(qn_handle h);
 #define QN_KERNEL_ROW_BULK 6     /* row refresh, fed and landed by bulk copies */
 #define QN_KERNEL_FP64_PRODUCTS 0x100
 QN_API int32_t qn_last_gram_kernel(qn_handle h);
+
+/*
+ * 1 if the most recent step whose results were fetched to the host (j_out or sigma_out non-NULL, or qn_status_sync)
+ * found a retained sigma_k too small for the accuracy of the Gram pass behind it AND could not repeat that pass
+ * itself, else 0.  Only qn_update_from_gram can leave it set (qn_update, qn_update_host and qn_apply_hinv repeat
+ * the pass on the device, see qn_update): the Gram it is given was summed by the caller, e.g. over the ranks of an
+ * n-sharded step.  The remedy is the caller's: select QN_GRAM_PATH_FP64, call qn_gram again on every rank, sum, and
+ * repeat the step (sigma and j are the same on every rank, so every rank sees the same flag).
+ */
+QN_API int32_t qn_precision_flag(qn_handle h);
 
 /* Jacobi sweeps used by the most recent step whose results were fetched to the host (j_out or
  * sigma_out non-NULL, or qn_status_sync), else -1. */

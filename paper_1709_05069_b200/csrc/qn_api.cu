@@ -56,6 +56,8 @@ struct qn_ctx {
     int32_t last_sweeps;
     int32_t last_kernel;  // QN_KERNEL_* of the most recent Gram or row pass
     int32_t redo_kernel;  // QN_KERNEL_* of the fp64 repeat pass that the most recent step enqueued (0: none)
+    int32_t gram_call_kernel;  // QN_KERNEL_* of the most recent qn_gram call on this handle (0: none yet)
+    int32_t precision_flag;    // bit 0 of the result block's redo word as last fetched
 };
 
 static int g_sm_count_cache[64];
@@ -139,6 +141,7 @@ qn_status fetch_result(qn_handle h, cudaStream_t st, int32_t* j_out, double* sig
     h->last_sweeps = h->host_result->sweeps;
     h->last_tau = h->host_result->tau_eff;
     if ((h->host_result->redo & 2) && h->redo_kernel) h->last_kernel = h->redo_kernel;  // the fp64 repeat pass ran
+    h->precision_flag = h->host_result->redo & 1;
     return static_cast<qn_status>(h->host_result->status);
 }
 
@@ -423,6 +426,10 @@ extern "C" qn_status qn_update_from_gram(qn_handle h, const void* theta, const v
     p.m = h->m;
     p.source = QN_SRC_SUMMED;
     p.raw_gram = const_cast<double*>(gram);  // read only in this mode
+    // If this handle's qn_gram produced the buffer (the n-sharded step), the solve can still judge the spectrum against
+    // that pass's accuracy; it cannot repeat the pass (the sum over the ranks is the caller's), so it only raises the
+    // flag that qn_precision_flag returns.
+    p.redo_coeff = h->gram_call_kernel ? qn_gram_error_coeff(h->gram_call_kernel, h->dtype, h->n, lambda) : 0.0;
     p.tau = tau;
     p.lambda = lambda;
     p.coef = h->coef;
@@ -540,6 +547,7 @@ extern "C" qn_status qn_gram(qn_handle h, const void* g, double* gram_out, void*
         p.lambda = 1.0;
         p.coef = h->coef;
         p.result = h->result;
+        h->gram_call_kernel = h->last_kernel;
         KernelTimer t(h, st, QN_TIME_SOLVE);
         if (qn_launch_solve(p, st, &h->last_launches) != cudaSuccess) s = QN_ERR_CUDA;
     }
@@ -746,6 +754,7 @@ extern "C" int32_t qn_last_launches(qn_handle h) { return h ? h->last_launches :
 extern "C" int64_t qn_total_launches(qn_handle h) { return h ? h->total_launches : 0; }
 extern "C" int32_t qn_last_sweeps(qn_handle h) { return h ? h->last_sweeps : -1; }
 extern "C" int32_t qn_last_gram_kernel(qn_handle h) { return h ? h->last_kernel : QN_KERNEL_NONE; }
+extern "C" int32_t qn_precision_flag(qn_handle h) { return h ? h->precision_flag : 0; }
 
 extern "C" qn_status qn_timing_begin(qn_handle h, int32_t max_kernels) {
     if (!h || max_kernels < 1 || max_kernels > (1 << 20)) return QN_ERR_INVALID;

@@ -29,7 +29,8 @@ EXPORTS = (
     "qn_set_rank_cap", "qn_set_sweep_limit", "qn_set_gram_path", "qn_set_tau_cap", "qn_last_tau", "qn_push",
     "qn_update_window", "qn_rebuild",
     "qn_window_alloc", "qn_window_theta", "qn_window_g", "qn_window_mark_full", "qn_update_host", "qn_status_sync",
-    "qn_last_launches", "qn_total_launches", "qn_last_sweeps", "qn_last_gram_kernel", "qn_timing_begin",
+    "qn_last_launches", "qn_total_launches", "qn_last_sweeps", "qn_last_gram_kernel", "qn_precision_flag",
+    "qn_timing_begin",
     "qn_timing_end",
     "qn_gram_static", "qn_selftest_bounded_wait",
 )
@@ -86,6 +87,7 @@ def lib() -> ctypes.CDLL:
         L.qn_total_launches.argtypes, L.qn_total_launches.restype = [vp], i64
         L.qn_last_sweeps.argtypes, L.qn_last_sweeps.restype = [vp], i32
         L.qn_last_gram_kernel.argtypes, L.qn_last_gram_kernel.restype = [vp], i32
+        L.qn_precision_flag.argtypes, L.qn_precision_flag.restype = [vp], i32
         L.qn_gram_static.argtypes, L.qn_gram_static.restype = [i64, i32, i32, vp, vp, vp], i32
         L.qn_timing_begin.argtypes, L.qn_timing_begin.restype = [vp, i32], i32
         L.qn_timing_end.argtypes, L.qn_timing_end.restype = [vp, vp, vp], i32
@@ -117,6 +119,7 @@ class Handle:
 
     def __init__(self, ptr: int, n: int, m: int, dtype: torch.dtype, device: int = 0):
         self.ptr, self.n, self.m, self.dtype, self.device = ptr, n, m, dtype, device
+        self.gram_path = QN_GRAM_PATH_AUTO  # as last set through qn_set_gram_path
 
     def close(self):
         if self.ptr:
@@ -238,6 +241,7 @@ def qn_set_gram_path(h: Handle, path: int) -> None:
     """``QN_GRAM_PATH_AUTO`` (default), ``QN_GRAM_PATH_PLAIN_ALU`` (register-fed plain-ALU Gram kernels only) or
     ``QN_GRAM_PATH_FP64`` (those kernels with fp64 products and sums whatever n)."""
     _check(lib().qn_set_gram_path(h.ptr, int(path)), "qn_set_gram_path")
+    h.gram_path = int(path)
 
 
 def qn_set_tau_cap(h: Handle, on: bool) -> None:
@@ -306,16 +310,33 @@ def qn_update_sharded(h: Handle, theta: torch.Tensor, g: torch.Tensor, tau: floa
     rank the all-reduce still runs (it is the identity).
 
     The collective is ordered against torch's CURRENT stream, so the three calls run with ``stream`` made current:
-    the all-reduce then sits between the Gram pass and the step on the same stream."""
+    the all-reduce then sits between the Gram pass and the step on the same stream.
+
+    With ``want_host`` the step's precision flag is read as well (``qn_precision_flag``): if the spectrum has a
+    retained mode too small for the reduced-precision Gram pass, the three calls are repeated once with the handle on
+    ``QN_GRAM_PATH_FP64``.  sigma and j are identical on every rank, so all ranks repeat together.  Without
+    ``want_host`` nothing is read back and nothing is repeated."""
     import torch.distributed as dist
 
     if stream is None:
         stream = torch.cuda.current_stream()
-    with torch.cuda.stream(stream):
+
+    def three_calls():
         qn_gram(h, g, gram_buf, stream=stream)
         if dist.is_available() and dist.is_initialized():
             dist.all_reduce(gram_buf, op=dist.ReduceOp.SUM, group=group)
         return qn_update_from_gram(h, theta, g, gram_buf, tau, lam, theta_new, want_host=want_host, stream=stream)
+
+    with torch.cuda.stream(stream):
+        res = three_calls()
+        if want_host and lib().qn_precision_flag(h.ptr):
+            before = h.gram_path
+            qn_set_gram_path(h, QN_GRAM_PATH_FP64)
+            try:
+                res = three_calls()
+            finally:
+                qn_set_gram_path(h, before)
+        return res
 
 
 def qn_push(h: Handle, slot: int, theta_col: torch.Tensor, g_col: torch.Tensor, stream=None) -> None:

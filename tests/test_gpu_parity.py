@@ -734,3 +734,80 @@ def test_gram_paths_at_large_n(qn, dtype, m):
         guarded.check()
         C = guarded.view[: m * m].view(m, m).cpu().numpy()
         assert np.max(np.abs(C - Cref)) <= tol * scale, (path, np.max(np.abs(C - Cref)) / scale)
+
+
+# --------------------------------------------------------------------------- the certificate through the other calls
+@pytest.mark.parametrize("n", [(1 << 20) - 8, 1 << 20, (1 << 20) + 8])
+@pytest.mark.parametrize("m", [9, 16])
+def test_tensor_core_threshold(qn, n, m):
+    """Both sides of the size from which the tensor cores carry the Gram pass (2^20 columns, m > 8), fp32 storage, on
+    the gap variant at lambda = 1e-2 and 1e-3 (the second needs the fp64 repeat above the threshold)."""
+    for lam in (1e-2, 1e-3):
+        cfg = W.Config(53, n, m, "f32", -2, 2, 0, 0.01, 1e-4, 1.0, lam)
+        theta, g = W.generate(cfg, "cuda", gap_lam=lam, gap_scale=1.0)
+        expect = assert_gap(theta, g, lam)
+        check_against_oracle(qn, theta, g, 1.0, lam, "f32", expect_j=expect)
+        if n < (1 << 20):
+            assert run_gpu.last_kernel.startswith("tiled") and "fp64" in run_gpu.last_kernel
+        elif lam == 1e-2:
+            assert run_gpu.last_kernel.startswith("tcgen05")
+        else:
+            assert "fp64 products" in run_gpu.last_kernel
+
+
+def test_certificate_through_apply_hinv_and_host_entry(qn):
+    """The fp64 repeat also runs behind qn_apply_hinv and qn_update_host: lambda = 1e-3 on the tensor-core path."""
+    lam, m, n = 1e-3, 24, (1 << 22) + 64
+    cfg = W.Config(54, n, m, "f32", -2, 2, 0, 0.01, 1e-4, 1.0, lam)
+    theta, g = W.generate(cfg, "cuda", gap_lam=lam, gap_scale=1.0)
+    tb, gb = W.to_bits(theta), W.to_bits(g)
+    z = (0.5 * (g[1] - g[0]) + torch.randn(n, device="cuda", generator=torch.Generator(device="cuda").manual_seed(5))).contiguous()
+    out = torch.empty(n, device="cuda")
+    with qn.qn_create(n, m, torch.float32) as h:
+        j, sigma, status = qn.qn_apply_hinv(h, theta, g, lam, z, out)
+        assert "fp64 products" in h.last_gram_kernel and h.last_launches == 6
+        ref, jref = oracle.apply_hinv(tb, gb, lam, oracle.storage_to_f64(W.to_bits(z)))
+        assert status == 0 and j == jref
+        got = oracle.storage_to_f64(W.to_bits(out))
+        assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= TOL["f32"]
+        th_h, g_h = theta.cpu().pin_memory(), g.cpu().pin_memory()
+        out_h = torch.empty(n).pin_memory()
+        j, sigma, status = qn.qn_update_host(h, th_h, g_h, 1.0, lam, out_h)
+        assert "fp64 products" in h.last_gram_kernel
+        full = oracle.update(tb, gb, 1.0, lam)
+        assert status == 0 and j == full.j
+        sigma = np.array(sigma)
+        assert np.max(np.abs(sigma[:j] - full.sigma[:j]) / full.sigma[:j]) <= 1e-5
+        assert np.linalg.norm(out_h.double().numpy() - full.theta_new) / np.linalg.norm(full.theta_new) <= TOL["f32"]
+
+
+def test_sharded_step_repeats_in_fp64_when_the_spectrum_needs_it(qn):
+    """qn_update_from_gram cannot repeat a Gram pass that the caller summed; it raises qn_precision_flag instead and
+    qn_update_sharded repeats its three calls with fp64 products.  lambda = 1e-3 on the tensor-core path."""
+    lam, m, n = 1e-3, 32, 1 << 22
+    cfg = W.Config(55, n, m, "f32", -2, 2, 0, 0.01, 1e-4, 1.0, lam)
+    theta, g = W.generate(cfg, "cuda", gap_lam=lam, gap_scale=1.0)
+    ref = oracle.update(W.to_bits(theta), W.to_bits(g), 1.0, lam)
+    buf = torch.empty(m * m + m, dtype=torch.float64, device="cuda")
+    out = torch.empty(n, device="cuda")
+    L = qn.lib()
+    with qn.qn_create(n, m, torch.float32) as h:
+        # by hand: the flag comes up and the sigma of the tensor-core pass are outside the bar
+        qn.qn_gram(h, g, buf)
+        j, sigma, status = qn.qn_update_from_gram(h, theta, g, buf, 1.0, lam, out)
+        assert L.qn_precision_flag(h.ptr) == 1
+        sigma = np.array(sigma)
+        assert np.max(np.abs(sigma[:ref.j] - ref.sigma[:ref.j]) / ref.sigma[:ref.j]) > 1e-5
+        # the sharded step repeats by itself
+        j, sigma, status = qn.qn_update_sharded(h, theta, g, 1.0, lam, out, buf)
+        assert L.qn_precision_flag(h.ptr) == 0 and h.gram_path == qn.QN_GRAM_PATH_AUTO
+        sigma = np.array(sigma)
+        assert status == 0 and j == ref.j
+        assert np.max(np.abs(sigma[:j] - ref.sigma[:j]) / ref.sigma[:j]) <= 1e-5
+        got = oracle.storage_to_f64(W.to_bits(out))
+        assert np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL["f32"]
+        # a spectrum that does not need it: no flag
+        cfg2 = W.Config(55, n, m, "f32", -2, 2, 0, 0.01, 1e-4, 1.0, 1e-2)
+        theta2, g2 = W.generate(cfg2, "cuda", gap_lam=1e-2, gap_scale=1.0)
+        j, sigma, status = qn.qn_update_sharded(h, theta2, g2, 1.0, 1e-2, out, buf)
+        assert L.qn_precision_flag(h.ptr) == 0 and h.last_gram_kernel.startswith("tcgen05")
