@@ -282,7 +282,8 @@ QN_API int64_t qn_total_launches(qn_handle h);
 /*
  * Which kernel the most recent Gram pass of this handle was dispatched to (qn_update, qn_update_host, qn_gram,
  * qn_apply_hinv, qn_rebuild), or, after qn_push, which row-refresh kernel ran; QN_KERNEL_NONE before the first.
- * Benchmarks label their numbers with it.  QN_KERNEL_FP64_PRODUCTS is or-ed in when every product and sum of the
+ * Benchmarks label their numbers with it.  When a step repeated its Gram pass in fp64 (see qn_update), this reports
+ * the fp64 kernel once the step's results have been fetched to the host.  QN_KERNEL_FP64_PRODUCTS is or-ed in when every product and sum of the
  * pass was formed in fp64 (n below 2^22, and qn_rebuild).
  */
 #define QN_KERNEL_NONE 0
