@@ -197,3 +197,23 @@ def test_config4_full_size_by_permuted_tiling(qn, m):
         perm = W.period_permutation(p, q, seed, "cuda")
         assert not torch.equal(perm, perm0)
         assert torch.equal(out[q * p:(q + 1) * p].view(torch.int16), by_source[perm].view(torch.int16)), q
+
+
+def test_config2_full_size_with_the_fp64_repeat(qn):
+    """Config 2's shape and generator (n = 25.6 M, m = 32, fp32) in the gap variant at lambda = 1e-3: the retained modes
+    reach down to 3.75e-3 sigma_1, the tensor-core pass cannot deliver them, and the step repeats the Gram pass with
+    fp64 products on the device.  j and sigma from the oracle's full passes, theta_new on sampled columns."""
+    lam = 1e-3
+    cfg = W.CONFIGS[2]
+    theta, g = W.generate(cfg, "cuda", gap_lam=lam, gap_scale=1.0)
+    rng = np.random.default_rng(17)
+    idx = np.unique(np.concatenate([[0, 127, 128, cfg.n - 1, cfg.n - 129], rng.integers(0, cfg.n, 4096)])).astype(np.int64)
+    ref = oracle.update(W.to_bits(theta), W.to_bits(g), cfg.tau, lam, sample_idx=idx)
+    assert 2 < ref.j < cfg.m - 1 and ref.sigma[ref.j - 1] >= 2 * lam * ref.sigma[0] and ref.sigma[ref.j] <= lam * ref.sigma[0] / 2
+    out, j, sigma, status, launches = run_gpu(qn, theta, g, cfg.tau, lam)
+    assert status == 0 and launches == 5 and j == ref.j
+    assert "fp64 products" in run_gpu.last_kernel
+    assert np.max(np.abs(sigma - ref.sigma)) <= 1e-5 * ref.sigma[0]
+    assert np.max(np.abs(sigma[:j] - ref.sigma[:j]) / ref.sigma[:j]) <= 1e-5
+    got = oracle.storage_to_f64(W.to_bits(out))[idx]
+    assert np.linalg.norm(got - ref.theta_new) / np.linalg.norm(ref.theta_new) <= TOL["f32"]
