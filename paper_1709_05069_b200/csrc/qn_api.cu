@@ -576,12 +576,12 @@ extern "C" qn_status qn_push(qn_handle h, int32_t slot, const void* theta_col, c
     if (!h || !theta_col || !g_col || slot < -1 || slot >= h->m) return QN_ERR_INVALID;
     DeviceGuard guard(h->device);
     if (!guard.ok) return QN_ERR_CUDA;
+    if (!on_device(theta_col, h->device) || !on_device(g_col, h->device)) return QN_ERR_INVALID;
     qn_status s = ensure_window(h);
     if (s != QN_OK) return s;
     const size_t col_bytes = (size_t)h->n * h->elem, win_bytes = col_bytes * h->m;
     if (overlaps(theta_col, col_bytes, h->win_theta, win_bytes) || overlaps(g_col, col_bytes, h->win_g, win_bytes))
         return QN_ERR_INVALID;
-    if (!on_device(theta_col, h->device) || !on_device(g_col, h->device)) return QN_ERR_INVALID;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     begin_call(h, st);
     const bool oldest = slot < 0;
@@ -706,13 +706,21 @@ extern "C" qn_status qn_update_host(qn_handle h, const void* theta_host, const v
         }
     }
     if (!h->copy_stream) {
-        bool ok = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
-        ok = ok && cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) == cudaSuccess;
-        ok = ok && cudaEventCreateWithFlags(&h->ev_theta, cudaEventDisableTiming) == cudaSuccess;
-        if (!ok) {
+        cudaStream_t cs = nullptr;
+        cudaEvent_t e0 = nullptr, e1 = nullptr;
+        bool ok = cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&e0, cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&e1, cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) {  // leave the handle as it was
+            if (e1) cudaEventDestroy(e1);
+            if (e0) cudaEventDestroy(e0);
+            if (cs) cudaStreamDestroy(cs);
             cudaGetLastError();
             return QN_ERR_CUDA;
         }
+        h->copy_stream = cs;
+        h->ev_fork = e0;
+        h->ev_theta = e1;
     }
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     begin_call(h, st);
