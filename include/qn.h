@@ -26,7 +26,9 @@
  * only reads inputs and only writes the named outputs.  The handle owns its workspace.
  * Rows that start on 16-byte boundaries (base pointer 16-byte aligned and n * element size a
  * multiple of 16) take the vectorised path; anything else takes a slower element-wise path,
- * never an error.
+ * never an error.  For full speed let every row start on a 128-byte boundary (n a multiple of 32
+ * for fp32 storage, of 64 for bf16): rows that only meet the 16-byte rule were measured 8 to 15 %
+ * slower, because every request of a streaming pass then touches one more cache line.
  *
  * Streams.  `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  * Calls enqueue work on that stream and return without waiting unless they have to hand a HOST
