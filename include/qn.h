@@ -282,7 +282,7 @@ QN_API int32_t qn_last_launches(qn_handle h);
 QN_API int64_t qn_total_launches(qn_handle h);
 
 /*
- * Which kernel the most recent Gram pass of this handle was dispatched to (qn_update, qn_update_host, qn_gram,
+ * (The paper has no counterpart.)  Which kernel the most recent Gram pass of this handle was dispatched to (qn_update, qn_update_host, qn_gram,
  * qn_apply_hinv, qn_rebuild), or, after qn_push, which row-refresh kernel ran; QN_KERNEL_NONE before the first.
  * Benchmarks label their numbers with it.  When a step repeated its Gram pass in fp64 (see qn_update), this reports
  * the fp64 kernel once the step's results have been fetched to the host.  QN_KERNEL_FP64_PRODUCTS is or-ed in when every product and sum of the
@@ -299,7 +299,7 @@ QN_API int64_t qn_total_launches(qn_handle h);
 QN_API int32_t qn_last_gram_kernel(qn_handle h);
 
 /*
- * 1 if the most recent step whose results were fetched to the host (j_out or sigma_out non-NULL, or qn_status_sync)
+ * (The paper has no counterpart.)  1 if the most recent step whose results were fetched to the host (j_out or sigma_out non-NULL, or qn_status_sync)
  * found a retained sigma_k too small for the accuracy of the Gram pass behind it AND could not repeat that pass
  * itself, else 0.  Only qn_update_from_gram can leave it set (qn_update, qn_update_host and qn_apply_hinv repeat
  * the pass on the device, see qn_update): the Gram it is given was summed by the caller, e.g. over the ranks of an
