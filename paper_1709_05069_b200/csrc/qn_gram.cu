@@ -781,7 +781,7 @@ double qn_gram_error_coeff(int kernel, qn_dtype dtype, int64_t n, double lambda_
     switch (kernel & 0xff) {
         case QN_KERNEL_GRAM_TENSOR: return dtype == QN_F32 ? QN_REDO_COEFF_TC_F32 : QN_REDO_COEFF_TC_BF16;
         case QN_KERNEL_GRAM_BULK:
-            return (dtype == QN_BF16 && lambda_hint >= QN_REF0_MIN_LAMBDA ? QN_REDO_COEFF_REF0_AT_4M : QN_REDO_COEFF_ALU_AT_4M) * by_n;
+            return (dtype == QN_BF16 && lambda_hint >= QN_REF0_MIN_LAMBDA ? QN_REDO_COEFF_REF0_AT_4M : QN_REDO_COEFF_BULK_AT_4M) * by_n;
         case QN_KERNEL_GRAM_DIRECT:
         case QN_KERNEL_GRAM_TILED: return QN_REDO_COEFF_ALU_AT_4M * by_n;
     }

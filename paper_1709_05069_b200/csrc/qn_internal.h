@@ -94,12 +94,14 @@ struct qn_solve_params {
 // error of sigma_k = coefficient * (sigma_1 / sigma_k)^2 on inputs whose largest modes sit on few Workers):
 //   tensor cores: the fp32 accumulator truncates each product, a bias proportional to the chain length and
 //                 independent of n: 2e-9 for fp32 storage (chains of 8 instructions), 2e-8 for bf16 (16)
-//   fp32 products on the plain ALUs: unbiased, 2e-10 at n = 2^22 and falling as 1 / sqrt(n); the bulk-copy kernel
-//                 with Worker 0 as its reference 2e-9 at n = 2^22
+//   fp32 products on the plain ALUs: unbiased, 2e-10 at n = 2^22 (tiled and register-fed kernels) or 6e-10 (bulk-copy
+//                 kernel, which adds 64 columns per accumulator in fp32) and falling as 1 / sqrt(n); the bulk-copy
+//                 kernel with Worker 0 as its reference 2e-9 at n = 2^22
 #define QN_REDO_TRIGGER 2.5e-6
 #define QN_REDO_COEFF_TC_F32 2e-9
 #define QN_REDO_COEFF_TC_BF16 2e-8
 #define QN_REDO_COEFF_ALU_AT_4M 2e-10
+#define QN_REDO_COEFF_BULK_AT_4M 6e-10
 #define QN_REDO_COEFF_REF0_AT_4M 2e-9
 // path: QN_GRAM_PATH_* of qn.h (qn_set_gram_path).
 cudaError_t qn_launch_gram(qn_dtype dtype, const void* g, int64_t n, int m, bool raw, double* partials,
