@@ -2,7 +2,7 @@
 """Benchmark of the Server quasi-Newton step (arXiv 1709.05069, Section 2) on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--m M] [--impl ours|reference]
-                    [--shard n] [--no-per-config] [--gram-path auto|alu]
+                    [--shard n] [--no-per-config] [--gram-path auto|alu|fp64]
 
 One step = one pass of the whole hot path (Gram pass, solve, combine; for the asynchronous config the row refresh
 of one Write followed by the update) over one resident synthetic input.  Prints ONE JSON line: updates/s of the
@@ -550,8 +550,8 @@ def main():
     ap.add_argument("--n", type=int, default=None, help="override n (profiling on a small case)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--shard", default=None, choices=["n"], help="share ONE problem over the ranks by columns")
-    ap.add_argument("--gram-path", default="auto", choices=["auto", "alu"],
-                    help="alu: plain-ALU Gram kernels only (A/B runs)")
+    ap.add_argument("--gram-path", default="auto", choices=["auto", "alu", "fp64"],
+                    help="alu: plain-ALU Gram kernels only (A/B runs); fp64: those with fp64 products whatever n")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
@@ -598,7 +598,7 @@ def main():
     if args.warmup is None:
         args.warmup = max(3, min(20, args.steps // 10))
     args.warmup = max(args.warmup, 3)
-    gram_path = qn.QN_GRAM_PATH_PLAIN_ALU if args.gram_path == "alu" else qn.QN_GRAM_PATH_AUTO
+    gram_path = {"auto": qn.QN_GRAM_PATH_AUTO, "alu": qn.QN_GRAM_PATH_PLAIN_ALU, "fp64": qn.QN_GRAM_PATH_FP64}[args.gram_path]
 
     if args.shard:
         rc = run_sharded(args, cfg, qn, dev, rank, world, local, peak, peak_kind)

@@ -123,3 +123,21 @@ def test_sharded_gram_buffers_add_up_to_the_whole_problem():
     scale = np.abs(C).max()
     assert np.max(np.abs(res[0][: cfg.m ** 2] - whole[: cfg.m ** 2])) <= 1e-12 * scale
     assert np.max(np.abs(res[0][cfg.m ** 2:] - whole[cfg.m ** 2:])) <= 1e-12 * max(np.abs(w).max(), scale)
+
+
+def test_reference_arm_prints_the_contract_line():
+    """`bench.py --impl reference` needs no GPU: it times the oracle and prints one JSON line with the keys of the
+    benchmark contract (checked on the smallest configuration)."""
+    import json
+    import subprocess
+
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "0",
+                          "--steps", "2", "--warmup", "1"], capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["metric"] == "qn_update/s" and line["unit"] == "updates/s"
+    assert line["steps"] == 2 and line["warmup"] == 1 and line["higher_is_better"] is True and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
+    assert line["cpu_baseline"]["min"] <= line["cpu_baseline"]["median"] <= line["cpu_baseline"]["max"]
+    assert line["e2e"] == {"value": line["value"], "unit": "updates/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+    assert line["config"]["n"] == 4096 and line["config"]["m"] == 8 and line["gpu_launches"] == 0
