@@ -16,7 +16,7 @@
  * Layout.  All matrices are Worker-major: theta[m][n] and g[m][n], row k = Worker k, each row
  * contiguous (the transpose of the paper's n x m matrices).  Elements are fp32 or bf16
  * (qn_dtype).  Arithmetic: the Gram pass forms fp64 products below 2^22 parameters and fp32 products
- * (m <= 8) or tensor-core products of a bf16 hi/lo split (m > 8, from 2^20 parameters on) above, always
+ * (m <= 8) or tensor-core products of a bf16 hi/lo split (m > 8, from 2^17 parameters on) above, always
  * with fp64 accumulation across work items, and is repeated in fp64 when the spectrum needs it (see
  * qn_update); the m x m eigen-problem and the coefficients are fp64; the final combination is fp32 with
  * one round-to-nearest-even to the storage type when theta_new is written.
@@ -107,7 +107,7 @@ QN_API qn_status qn_destroy(qn_handle h);
  * lies within 1e-5 sigma_1 of lambda sigma_1; every sigma_k within 1e-5 sigma_1, the retained ones within a
  * relative 1e-5; theta_new within a relative L2 error of 1e-5 (fp32 storage) or 2e-3 (bf16 storage: the single
  * rounding of the output).  The first Gram pass is chosen from n, m, the storage type and lambda (fp64 products
- * below 2^22 parameters, or 2^20 with m > 8; fp32 or tensor-core products above), never from the data.
+ * below 2^22 parameters, or 2^17 with m > 8; fp32 or tensor-core products above), never from the data.
  * How the sigma figures are kept where the Gram pass rounds: fp32 products on the plain ALUs
  * (unbiased; the relative error of a retained sigma_k is about 2e-10 (sigma_1 / sigma_k)^2 at n = 2^22 and falls as
  * 1 / sqrt(n)), or for m > 8 the tensor cores, whose fp32 accumulator truncates each product: measured, a retained
@@ -210,7 +210,7 @@ QN_API qn_status qn_gram(qn_handle h, const void* g, double* gram_out, void* cud
  *      sigma are the same on every rank.
  *   gram         DEVICE, m*m + m doubles as written by qn_gram (or sums of such buffers), read only
  *   other arguments as for qn_update.  Errors as for qn_update.
- * Accuracy: that of the Gram it is given.  Above 2^22 parameters (2^20 with m > 8) qn_gram rounds its products (see
+ * Accuracy: that of the Gram it is given.  Above 2^22 parameters (2^17 with m > 8) qn_gram rounds its products (see
  * qn_update); this call checks the spectrum against that pass's accuracy like qn_update does, but cannot repeat
  * the pass: see qn_precision_flag.
  */

@@ -18,11 +18,12 @@ __host__ __device__ inline int qn_partial_len(int m) { return m * (m + 1) / 2 + 
 // needed for sigma to be good to 1e-5 * sigma_1 on near-null modes once n is a few million.
 #define QN_PRECISE_BELOW (int64_t(1) << 22)
 // The tensor-core Gram pass (m > 8) starts earlier: its error does not depend on n (the truncating accumulation is a
-// bias), a step checks it against the spectrum on the device and repeats the pass in fp64 where needed, and from
-// about a million columns on it is several times faster than the fp64 pass even though a CTA only gets a few dozen
-// stages.
+// bias), a step checks it against the spectrum on the device and repeats the pass in fp64 where needed, and it is
+// faster than the fp64 pass from a few ten thousand columns on even though a CTA then only gets a handful of stages
+// (measured, whole step, m = 32: 139 against 158 us at n = 2^17, 162 against 243 us at 2^19; below 2^17 the two are
+// within 5 % and the eigen-solve is nearly all of the step).
 #ifndef QN_TC_MIN_N
-#define QN_TC_MIN_N (int64_t(1) << 20)
+#define QN_TC_MIN_N (int64_t(1) << 17)
 #endif
 
 // Eigenvalues of the centred Gram below this fraction of the largest diagonal entry of the

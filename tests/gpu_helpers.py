@@ -42,10 +42,10 @@ def run_gpu(qn, theta, g, tau, lam):
 
 
 def step_launches(n, base=3, m=64):
-    """Kernels of one step: from 2^22 parameters on (2^20 with more than 8 Workers: tensor cores) the Gram pass has
+    """Kernels of one step: from 2^22 parameters on (2^17 with more than 8 Workers: tensor cores) the Gram pass has
     reduced precision, and unless lambda is so large that no retained mode can need it, the step enqueues a
     conditional fp64 repeat of the pass and of the solve (both return at once unless the spectrum asks for them)."""
-    return (base,) if n < ((1 << 20) if m > 8 else (1 << 22)) else (base, base + 2)
+    return (base,) if n < ((1 << 17) if m > 8 else (1 << 22)) else (base, base + 2)
 
 
 def _cudart():

@@ -737,17 +737,17 @@ def test_gram_paths_at_large_n(qn, dtype, m):
 
 
 # --------------------------------------------------------------------------- the certificate through the other calls
-@pytest.mark.parametrize("n", [(1 << 20) - 8, 1 << 20, (1 << 20) + 8])
+@pytest.mark.parametrize("n", [(1 << 17) - 8, 1 << 17, (1 << 17) + 8])
 @pytest.mark.parametrize("m", [9, 16])
 def test_tensor_core_threshold(qn, n, m):
-    """Both sides of the size from which the tensor cores carry the Gram pass (2^20 columns, m > 8), fp32 storage, on
+    """Both sides of the size from which the tensor cores carry the Gram pass (2^17 columns, m > 8), fp32 storage, on
     the gap variant at lambda = 1e-2 and 1e-3 (the second needs the fp64 repeat above the threshold)."""
     for lam in (1e-2, 1e-3):
         cfg = W.Config(53, n, m, "f32", -2, 2, 0, 0.01, 1e-4, 1.0, lam)
         theta, g = W.generate(cfg, "cuda", gap_lam=lam, gap_scale=1.0)
         expect = assert_gap(theta, g, lam)
         check_against_oracle(qn, theta, g, 1.0, lam, "f32", expect_j=expect)
-        if n < (1 << 20):
+        if n < (1 << 17):
             assert run_gpu.last_kernel.startswith("tiled") and "fp64" in run_gpu.last_kernel
         elif lam == 1e-2:
             assert run_gpu.last_kernel.startswith("tcgen05")

@@ -46,9 +46,9 @@ def test_static_gram_matches_handle_gram_twice(dtype, m, n):
         C = outs_static[-1][: m * m].reshape(m, m)
         w = outs_static[-1][m * m:]
         Cref = oracle.gram(W.to_bits(g))
-        # below 2^22 columns every product and sum is fp64; above, with m > 8, the tensor cores add in fp32 and
+        # below 2^17 columns (2^22 for m <= 8) every product and sum is fp64; above, with m > 8, the tensor cores add in fp32 and
         # truncate, which scales the whole Gram down by a few 1e-7 (harmless for sigma_k / sigma_1 and the update)
-        assert np.max(np.abs(C - Cref)) <= (2e-9 if n < (1 << 22) else 1e-6) * np.abs(Cref).max()
+        assert np.max(np.abs(C - Cref)) <= (2e-9 if (n < (1 << 17) or m <= 8) else 1e-6) * np.abs(Cref).max()
         assert np.array_equal(C, C.T)
         g64 = oracle.storage_to_f64(W.to_bits(g))
         gbar = g64.mean(0)
