@@ -141,3 +141,52 @@ def test_reference_arm_prints_the_contract_line():
     assert line["cpu_baseline"]["min"] <= line["cpu_baseline"]["median"] <= line["cpu_baseline"]["max"]
     assert line["e2e"] == {"value": line["value"], "unit": "updates/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     assert line["config"]["n"] == 4096 and line["config"]["m"] == 8 and line["gpu_launches"] == 0
+
+
+def _slice_rank_main(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world),
+                      LOCAL_RANK=str(rank))
+    import torch.distributed as dist
+
+    import workloads as W
+    from paper_1709_05069_b200 import qn
+
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    # what bench.py --shard n does before its first step, on the CPU: every rank forms its share of the low-rank
+    # products, the shares are added over the ranks, and every rank generates only its own column slice
+    cfg = W.CONFIGS[4].with_shape(n=3 * W.CHUNK + 4104, m=6)
+    nchunks = (cfg.n + W.CHUNK - 1) // W.CHUNK
+    c0, c1 = nchunks * rank // world, nchunks * (rank + 1) // world
+    wt = W.low_rank_products(cfg, "cpu", min(c0 * W.CHUNK, cfg.n), min(c1 * W.CHUNK, cfg.n))
+    dist.all_reduce(wt)
+    b, e = qn.shard_columns(cfg.n, world, rank)
+    theta, g = W.generate_slice(cfg, "cpu", b, e, wt)
+    out[rank] = (b, e, W.to_bits(theta), W.to_bits(g))
+    dist.destroy_process_group()
+
+
+def test_sharded_input_generation_matches_the_whole_problem():
+    """Two ranks that each generate only their column slice (the low-rank part of A couples the columns, so its
+    r x m products are added over the ranks first) hold exactly the bits of the whole problem's generator."""
+    import numpy as np
+
+    sys.path.insert(0, ROOT)
+    import workloads as W
+
+    world, port = 2, _free_port()
+    with mp.get_context("spawn").Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_slice_rank_main, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    cfg = W.CONFIGS[4].with_shape(n=3 * W.CHUNK + 4104, m=6)
+    theta, g = W.generate(cfg, "cpu")
+    tb, gb = W.to_bits(theta), W.to_bits(g)
+    assert res[0][0] == 0 and res[0][1] == res[1][0] and res[1][1] == cfg.n
+    for r in range(world):
+        b, e, ts, gs = res[r]
+        assert np.array_equal(ts, tb[:, b:e])
+        # the products are added in another order than in the one-process generator: the gradient may differ by one
+        # rounding of the fp32 sum, i.e. by at most one unit of the storage type in a few places
+        diff = np.abs(gs.astype(np.int64) - gb[:, b:e].astype(np.int64))
+        assert diff.max() <= 1 and (diff > 0).mean() < 1e-3
