@@ -577,11 +577,6 @@ def main():
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     if world > 1 or args.shard:
-        if args.shard:
-            # the sharded step has a real exchange: leave NCCL's own account of the communicator it builds (rings or
-            # trees, NVLS or not) in the log, on stderr
-            os.environ.setdefault("NCCL_DEBUG", "INFO")
-            os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
         import torch.distributed as dist
 
         if "MASTER_ADDR" in os.environ and "RANK" in os.environ:
